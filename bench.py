@@ -1,0 +1,329 @@
+#!/usr/bin/env python
+"""Throughput of libersd's verify path on synthetic Zipf-shaped logits.
+
+A step is one pass of the whole hot path (race variables, race keys, draft and
+target winners, accepted-prefix scan: ONE kernel launch) over one batch.  The
+default workload is the serving-scale sequence configuration (B=256, k=5,
+V=128256, bf16, per-row Zipf exponents, per-sequence temperatures); three
+distinct input sets are rotated so that every launch reads data the previous one
+did not touch (each set, 722 MB, is larger than the 126 MB L2 anyway).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c5|c3|c4|c2] [--impl reference]
+
+With N > 1 (under torch.distributed.run) every rank runs an independent replica
+on its own GPU -- the path has no exchange step -- and rank 0 reports the total.
+`--impl reference` times the CPU oracle, as it stands, on the host cores.
+Prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "race-verified logit rows/s at V=128256 bf16 (B*(k+1) rows)"
+UNIT = "rows/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        inside = [r for t, r in self.rows if t0 - 0.05 <= t <= t1 + 0.15] or [r for _, r in self.rows]
+        sm, smax, reasons = [], [], set()
+        for r in inside:
+            try:
+                sm.append(float(r[0]))
+                smax.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                 r[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None, "reasons": sorted(reasons),
+                "samples": len(inside)}
+
+
+def algorithmic_bytes(w, inp):
+    """Bytes one verify launch must read: every target row, every draft row that has children."""
+    es = inp["target"].element_size()
+    if w.is_tree:
+        parent = inp["parent"]
+        internal = len({p for p in parent if p >= 0})
+        rows = w.B * (w.rows_target + internal)
+    else:
+        rows = w.B * (w.rows_target + w.k)
+    return rows * w.V * es
+
+
+def oracle_rate(w, inp, n_seq, reps=1):
+    """rows/s of the CPU oracle on the first n_seq sequences of inp (host copies made here)."""
+    import oracle
+    from paper_2504_15475_b200 import workloads as wl
+    tgt = wl.as_numpy_logits(inp["target"][:n_seq])
+    drf = wl.as_numpy_logits(inp["draft"][:n_seq])
+    seeds = wl.seeds_as_u64(inp["seeds"][:n_seq])
+    temps = None if inp.get("temps") is None else inp["temps"][:n_seq].cpu().numpy()
+    best = None
+    for _ in range(reps):
+        t0 = time.perf_counter()
+        if w.is_tree:
+            oracle.verify_tree(tgt, drf, inp["parent"], seeds, T=inp["T"], temps=temps)
+        else:
+            oracle.verify(tgt, drf, seeds, T=inp["T"], temps=temps)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    return n_seq * w.rows_target / best, best, oracle.max_threads()
+
+
+def run_reference(args, w):
+    """The oracle as the reference arm: rank 0 only, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2504_15475_b200 import workloads as wl
+    n_seq = max(1, min(w.B, args.ref_seqs))
+    inp = wl.make_inputs(wl.scaled(w, B=n_seq), call=0)
+    for _ in range(args.warmup):
+        oracle_rate(w, inp, n_seq)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_rate(w, inp, n_seq)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = n_seq * w.rows_target / dt
+    sample = "%d of %d sequences of %s per step (%d logit rows)" % (n_seq, w.B, w.name,
+                                                                     n_seq * (w.rows_target + w.k))
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w, "oracle sample"),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.max_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def workload_config(w, l2_note):
+    return {"workload": "%s: B=%d k=%d V=%d %s %s" % (w.name, w.B, w.k, w.V, w.dtype,
+                                                     "tree" if w.is_tree else "sequence"),
+            "B": w.B, "k": w.k, "V": w.V, "rows_per_step": w.B * w.rows_target,
+            "l2": l2_note, "parallelism": "replicas only (no exchange step)"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default="c5")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sets", type=int, default=3, help="distinct input sets rotated between launches")
+    ap.add_argument("--e2e-steps", type=int, default=4)
+    ap.add_argument("--ref-seqs", type=int, default=64, help="sequences per oracle step (reference arm)")
+    ap.add_argument("--cpu-seqs", type=int, default=96, help="sequences of the oracle sample (cpu_baseline)")
+    ap.add_argument("--split", type=int, default=0, help="thread blocks per row (0: library default)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--sigma", type=float, default=None)
+    ap.add_argument("--temperature", type=float, default=None)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    from paper_2504_15475_b200 import workloads as wl
+    w = wl.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    from paper_2504_15475_b200 import binding
+    binding.lib()  # fail loudly if the CUDA library is missing
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    # ---- inputs: resident in HBM before the timed region; every rank has its own replica
+    sets = []
+    for s in range(max(1, args.sets)):
+        sets.append(wl.make_inputs(w, call=rank * 100 + s, device="cuda", sigma=args.sigma,
+                                   T=args.temperature))
+    D = w.k if not w.is_tree else binding.ersd_tree_depth(w.parent)
+    tokens = torch.empty(w.B, D + 1, dtype=torch.int32, device="cuda")
+    accept = torch.empty(w.B, dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def opts_for(inp):
+        kw = dict(split_v=args.split)
+        if inp.get("temps") is not None:
+            kw.update(temps=inp["temps"], temp_strides=(inp["temps"].stride(0), inp["temps"].stride(1)))
+        return binding.make_opts(**kw)
+
+    all_opts = [opts_for(inp) for inp in sets]
+
+    def step(i):
+        inp = sets[i % len(sets)]
+        if w.is_tree:
+            binding.ersd_verify_tree(inp["target"], inp["draft"], inp["parent"], inp["seeds"], inp["T"],
+                                     tokens, accept, all_opts[i % len(sets)], stream)
+        else:
+            binding.ersd_verify(inp["target"], inp["draft"], inp["seeds"], inp["T"], tokens, accept,
+                                all_opts[i % len(sets)], stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.25)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_wall0 = time.time()
+    ev0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    ev1.record(stream)
+    barrier()
+    t_wall1 = time.time()
+    clocks = sampler.stop(t_wall0, t_wall1)
+    ms_total = ev0.elapsed_time(ev1)
+    if dist is not None:
+        t = torch.tensor([ms_total], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    rows_per_step = w.B * w.rows_target
+    value = world * rows_per_step / (ms_step * 1e-3)
+    mean_accept = float(accept.float().mean().item())
+
+    # ---- roofline of the one kernel a step launches
+    peak, peak_kind = load_peaks()
+    alg_bytes = algorithmic_bytes(w, sets[0])
+    achieved = alg_bytes / (ms_step * 1e-3) / 1e9
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "traffic_per_index.json")
+    if os.path.exists(tpath):
+        with open(tpath) as f:
+            tj = json.load(f)
+        traffic = tj["dram_bytes_per_algorithmic_byte"] * alg_bytes
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": traffic, "peak_kind": peak_kind + " copy bandwidth",
+                "algorithmic_bytes_per_launch": alg_bytes, "kernel": "ersd_race_kernel<bf16>",
+                "kernel_ms": ms_step}
+
+    # ---- end to end: host buffers in pinned memory, copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        h = sets[0]
+        host_t = h["target"].cpu().pin_memory()
+        host_d = h["draft"].cpu().pin_memory()
+        host_s = h["seeds"].cpu().pin_memory()
+        host_temps = None if h.get("temps") is None else h["temps"].cpu().pin_memory()
+        for _ in range(2):
+            binding.verify_host(host_t, host_d, host_s, h["T"], temps=host_temps, parent=h.get("parent"))
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            tok_h, acc_h = binding.verify_host(host_t, host_d, host_s, h["T"], temps=host_temps,
+                                               parent=h.get("parent"))
+        torch.cuda.synchronize()
+        dt = (time.perf_counter() - t0) / args.e2e_steps
+        if dist is not None:
+            t = torch.tensor([dt], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        h2d = sum(x.numel() * x.element_size() for x in (host_t, host_d, host_s) if x is not None)
+        if host_temps is not None:
+            h2d += host_temps.numel() * 4
+        e2e = {"value": world * rows_per_step / dt, "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": tok_h.numel() * 4 + acc_h.numel() * 4, "ms_per_step": dt * 1e3,
+               "steps": args.e2e_steps}
+
+    # ---- the oracle on the host cores, on a bounded sample of the same workload (rank 0, N = 1)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        n_seq = max(1, min(w.B, args.cpu_seqs))
+        rate, secs, cores = oracle_rate(w, sets[0], n_seq)
+        cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": "first %d of %d sequences of input set 0 (%d logit rows), one pass, %.2f s" % (
+                   n_seq, w.B, n_seq * (w.rows_target + w.k), secs)}
+
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32 screen + f64 decision, u32 Philox", "data": "synthetic",
+            "config": workload_config(w, "inputs larger than L2; %d input sets rotated" % len(sets)),
+            "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps, "roofline": roofline,
+            "cpu_baseline": cpu, "mean_accept_len": mean_accept}))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,185 @@
+/*
+ * libersd -- exponential-race speculative decoding (ERSD) on one B200 (sm_100a).
+ *
+ * The library computes the data-parallel step of ERSD: for every draft and
+ * target logit row, the winner (or the first c arrivals) of an exponential
+ * race over the vocabulary, with the draft row and the target row of the same
+ * position sharing one realisation of the race variables, and from those
+ * winners the accepted prefix and the extra token.
+ *
+ * The race (Section 3 of the paper, "Exponential Races"): every token i gets
+ * e_i ~ Exp(1); the winner under a law p is argmin_i e_i / p_i and is
+ * distributed as p.  With p = softmax(logit / T) the library evaluates the
+ * equivalent log form
+ *
+ *     key_i = ln e_i - logit_i / T,        winner = argmin_i key_i,
+ *
+ * which needs no softmax (ln(e_i/p_i) = key_i + ln Z, Z free of i).  The paper
+ * names no random generator; here e_i = -log1p(-w_i), w_i = (x_i + 1/2) 2^-32,
+ * with x_i word (i & 3) of Philox4x32-10 (Salmon et al. 2011) under key
+ * (low, high 32 bits of seeds[b]) and counter (i >> 2, position, sequence id,
+ * 0).  position = pos_offsets[b] + r (r = row index, or node id in a tree);
+ * sequence id = b unless opts->seq_ids is given.  Exact key ties go to the
+ * lowest token id.  A NaN logit counts as -inf; -inf never wins; a row in
+ * which no token has positive probability yields token -1.
+ *
+ * Conventions for every call
+ *   - Unless stated otherwise every data pointer is a DEVICE pointer to memory
+ *     owned by the caller; the library never frees or keeps caller memory.
+ *   - Logit tensors are row-major with the vocabulary contiguous.  Rows are
+ *     `ld` elements apart (opts->ld_*; 0 means V) and row (b, r) starts at
+ *     element (b * rows_per_sequence + r) * ld.  16-byte aligned rows take
+ *     the vectorised path; other alignments are accepted and take a slower
+ *     scalar path.
+ *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t, NULL = default
+ *     stream) and never synchronise.  The return value is a host-side status:
+ *     argument errors are found before anything is launched, launch errors
+ *     are reported as ERSD_ECUDA (see ersd_last_cuda_error).
+ *   - T is the temperature of every row unless opts->temps is given.  It must
+ *     be finite and >= 0; T == 0 selects greedy decoding (key_i = -logit_i,
+ *     no randomness).  A per-row temperature that is negative or not finite
+ *     makes that row yield token -1.
+ *   - Scratch memory: calls that split rows over several thread blocks, and
+ *     every verify call, exchange partial results through a workspace.  Give
+ *     one in opts->workspace (size from ersd_workspace_bytes, zeroed once
+ *     with ersd_workspace_init; the library leaves it zeroed) or pass none
+ *     and the library keeps a private one per device, (re)allocated with
+ *     cudaMalloc when a call needs more than it holds.  Two calls that may
+ *     overlap on the GPU must not share a workspace.
+ *   - Randomness contract: a (seed, sequence id, position) triple must not be
+ *     reused for two EMITTED tokens.  Reusing the positions of a rejected
+ *     speculation in the next round is fine: what is emitted depends only on
+ *     races at positions up to the first disagreement.
+ */
+#ifndef ERSD_H_
+#define ERSD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { ERSD_F32 = 0, ERSD_BF16 = 1 } ersd_dtype;
+
+typedef enum {
+  ERSD_OK = 0,
+  ERSD_EINVAL = -1,       /* bad argument (null pointer, size out of range, bad T, bad tree) */
+  ERSD_EALIGN = -2,       /* pointer not aligned to its element size */
+  ERSD_EUNSUPPORTED = -3, /* size beyond a compiled limit (see ERSD_MAX_*) */
+  ERSD_ECUDA = -4,        /* a CUDA runtime call failed; see ersd_last_cuda_error() */
+  ERSD_EWORKSPACE = -5    /* opts->workspace given but too small */
+} ersd_status;
+
+#define ERSD_MAX_TOP_C 32   /* arrivals per race (children per tree node, opts->top_c) */
+#define ERSD_MAX_ROWS 256   /* rows per sequence: k + 1, N + 1 */
+#define ERSD_MAX_SPLIT 32   /* thread blocks sharing one row */
+
+/* Optional arguments.  Pass NULL for defaults.  Set struct_size = sizeof(ersd_opts). */
+typedef struct ersd_opts {
+  uint32_t struct_size;
+  uint32_t top_c;          /* ersd_race_sample: arrivals per row, 0 or 1 = winner only */
+  uint32_t split_v;        /* thread blocks per row; 0 = chosen by the library */
+  uint32_t reserved0;
+  int64_t ld_target;       /* row stride in elements of target_logits / logits; 0 = V */
+  int64_t ld_draft;        /* row stride in elements of draft_logits; 0 = V */
+  const float* temps;      /* device; temperature of row (b, r) = temps[b*temp_stride_b + r*temp_stride_r] */
+  int64_t temp_stride_b;
+  int64_t temp_stride_r;
+  const uint32_t* seq_ids;     /* device [B]; NULL: sequence id = b */
+  const uint32_t* pos_offsets; /* device [B]; NULL: 0 */
+  int32_t* out_draft_tok;  /* device, nullable.  verify: [B, k], entry j = token drafted at position j.
+                              verify_tree: [B, N+1], entry n = token drafted at node n (entry 0 = -1). */
+  float* out_draft_key;    /* device, nullable, same shape: race key of that drafted token */
+  int32_t* out_target_tok; /* device, nullable, [B, k+1] / [B, N+1]: target winner of every row */
+  float* out_target_key;   /* device, nullable, same shape: its race key */
+  int32_t* out_path;       /* device, nullable, verify_tree: [B, D+1] accepted node ids, -1 padded */
+  float* out_key;          /* device, nullable, ersd_race_sample: [B, R, c] keys of the arrivals */
+  void* workspace;         /* device scratch or NULL (library-owned) */
+  size_t workspace_bytes;
+} ersd_opts;
+
+/*
+ * Race sampling (Section 3; the drafting lines of Algorithms 2 and 5).
+ * For every sequence b < B and row r < R: out_tok[b, r, 0..c) = the first c
+ * arrivals (c = max(1, opts->top_c), ascending key; -1 where fewer than c
+ * tokens have positive probability) of the race of position
+ * pos_offsets[b] + r under softmax(logits[b, r, :] / T).  The ordered
+ * arrivals are a sample without replacement, which is how batch and tree
+ * drafting pick sibling tokens.
+ *   logits  device [B, R, V] of dtype dt       seeds   device [B] uint64
+ *   out_tok device [B, R, c] int32
+ * Errors: ERSD_EINVAL for null pointers, B, R, V < 1 or B * R beyond 2^31 - 1,
+ * T < 0 or not finite; ERSD_EUNSUPPORTED for c > ERSD_MAX_TOP_C or
+ * V > 0x7FFF0000; ERSD_EALIGN.
+ */
+int ersd_race_sample(const void* logits, ersd_dtype dt, const uint64_t* seeds, int B, int R, int V,
+                     float T, int32_t* out_tok, const ersd_opts* opts, void* cuda_stream);
+
+/*
+ * Sequence ERSD verification (Algorithm 2, extended to k drafted positions as
+ * Section 3 describes: one race per position, accept in order until the first
+ * disagreement).  For every sequence b and position j:
+ *   draft_tok[j]  = winner of race (b, j) under draft row j            (j < k)
+ *   target_tok[j] = winner of the SAME race under target row j         (j <= k)
+ *   L = first j < k with draft_tok[j] != target_tok[j] (or target_tok[j] = -1), else k
+ *   out_tokens[b, 0..L] = target_tok[0..L], out_tokens[b, j > L] = -1,
+ *   out_accept_len[b] = L   (L + 1 tokens are emitted, between 1 and k + 1).
+ *   target_logits device [B, k+1, V]    draft_logits device [B, k, V] (may be NULL when k = 0)
+ *   seeds device [B] uint64   out_tokens device [B, k+1] int32   out_accept_len device [B] int32
+ * Everything runs in one kernel launch.  Errors as above; k + 1 > ERSD_MAX_ROWS
+ * is ERSD_EUNSUPPORTED.
+ */
+int ersd_verify(const void* target_logits, const void* draft_logits, ersd_dtype dt,
+                const uint64_t* seeds, int B, int k, int V, float T, int32_t* out_tokens,
+                int32_t* out_accept_len, const ersd_opts* opts, void* cuda_stream);
+
+/*
+ * Tree ERSD verification (Algorithm 5; batch drafting is the depth-1 tree).
+ * The draft tree has nodes 0..N, node 0 the root (the current context).
+ * `parent` is a HOST array [N+1] with parent[0] = -1 and 0 <= parent[n] < n.
+ * Siblings are ordered by node id; the sibling of rank r (0-based) is taken
+ * to carry the (r+1)-th arrival of its parent's race under the parent's
+ * draft row.  Node n's race is the race of position pos_offsets[b] + n.
+ * Walk: cur = root; emit the winner of cur's race under target row cur; move
+ * to the child that drafted this token; stop when there is none.
+ *   target_logits device [B, N+1, V], row n = target law after the path to node n
+ *   draft_logits  device [B, N+1, V], row n = draft law after that path; rows of
+ *                 leaves are never read
+ *   out_tokens device [B, D+1] int32 (-1 padded), D = ersd_tree_depth(parent, N)
+ *   out_accept_len device [B] int32 = number of drafted tokens accepted
+ * Errors as above; a malformed parent array is ERSD_EINVAL; N + 1 > ERSD_MAX_ROWS
+ * or a node with more than ERSD_MAX_TOP_C children is ERSD_EUNSUPPORTED.
+ */
+int ersd_verify_tree(const void* target_logits, const void* draft_logits, ersd_dtype dt,
+                     const int32_t* parent, const uint64_t* seeds, int B, int N, int V, float T,
+                     int32_t* out_tokens, int32_t* out_accept_len, const ersd_opts* opts,
+                     void* cuda_stream);
+
+/* Depth (longest root-to-leaf edge count) of a HOST parent array, or -1 if it is malformed. */
+int ersd_tree_depth(const int32_t* parent, int N);
+
+/*
+ * Race keys of one row, for diagnostics and tests (Section 3, key_i as above,
+ * natural-log units): out_keys[i], i < V, device float32.
+ *   mode 0: the double-precision evaluation the library uses to decide winners;
+ *   mode 1: the single-precision screening value it uses to discard losers
+ *           (within about 1e-3 of mode 0 for |key| up to a few hundred).
+ */
+int ersd_row_keys(const void* row_logits, ersd_dtype dt, int V, float T, uint64_t seed,
+                  uint32_t seq_id, uint32_t position, int mode, float* out_keys, void* cuda_stream);
+
+/* Bytes of scratch that any call with these sizes can need. */
+size_t ersd_workspace_bytes(int B, int rows_per_seq);
+/* Zero a caller-owned workspace (needed once, before its first use). */
+int ersd_workspace_init(void* workspace, size_t bytes, void* cuda_stream);
+
+const char* ersd_status_string(int status);
+int ersd_last_cuda_error(void); /* cudaError_t of the last failing runtime call on this thread */
+int ersd_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ERSD_H_ */

@@ -1,0 +1,106 @@
+// Scalar building blocks of the race: Philox4x32-10, the Exp(1) transform and
+// the two evaluations of a race key.  Plain C++ when compiled without nvcc so
+// that a host harness can check the error bounds that the kernels rely on.
+#pragma once
+#include <math.h>
+#include <stdint.h>
+
+#if defined(__CUDACC__)
+#define ERSD_HD __host__ __device__ __forceinline__
+#else
+#define ERSD_HD inline
+#endif
+
+namespace ersd {
+
+constexpr uint32_t kPhiloxM0 = 0xD2511F53u;
+constexpr uint32_t kPhiloxM1 = 0xCD9E8D57u;
+constexpr uint32_t kPhiloxW0 = 0x9E3779B9u;
+constexpr uint32_t kPhiloxW1 = 0xBB67AE85u;
+
+ERSD_HD void mulhilo(uint32_t a, uint32_t b, uint32_t& hi, uint32_t& lo) {
+  const uint64_t p = (uint64_t)a * (uint64_t)b;
+  hi = (uint32_t)(p >> 32);
+  lo = (uint32_t)p;
+}
+
+// Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11): ten rounds of two
+// 32x32->64 products and a word shuffle, the key advancing by the Weyl
+// constants between rounds.
+ERSD_HD void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
+                           uint32_t k1, uint32_t out[4]) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    uint32_t hi0, lo0, hi1, lo1;
+    mulhilo(kPhiloxM0, c0, hi0, lo0);
+    mulhilo(kPhiloxM1, c2, hi1, lo1);
+    c0 = hi1 ^ c1 ^ k0;
+    c1 = lo1;
+    c2 = hi0 ^ c3 ^ k1;
+    c3 = lo0;
+    k0 += kPhiloxW0;
+    k1 += kPhiloxW1;
+  }
+  out[0] = c0;
+  out[1] = c1;
+  out[2] = c2;
+  out[3] = c3;
+}
+
+// The 32-bit word of token i in the race keyed by (seed, seq_id, position).
+ERSD_HD uint32_t token_word(uint64_t seed, uint32_t seq_id, uint32_t position, uint32_t i) {
+  uint32_t o[4];
+  philox4x32_10(i >> 2, position, seq_id, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), o);
+  return o[i & 3u];
+}
+
+ERSD_HD float lg2_fast(float a) {
+#if defined(__CUDA_ARCH__)
+  float r;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(a));
+  return r;
+#else
+  return log2f(a);
+#endif
+}
+
+// ln(e) for e = -log1p(-w), w = (x + 1/2) 2^-32, in double precision.  This is
+// the value that decides winners.
+ERSD_HD double exact_ln_e(uint32_t x) {
+  const double w = ((double)x + 0.5) * (1.0 / 4294967296.0);
+  return log(-log1p(-w));
+}
+
+// Exact race key in natural-log units; greedy rows (T == 0) use -z.
+ERSD_HD double exact_key(uint32_t x, float z, float T) {
+  if (z != z) return (double)INFINITY;  // NaN logit counts as -inf
+  if (T == 0.0f) return -(double)z;
+  return exact_ln_e(x) - (double)z / (double)T;
+}
+
+// Screening value: log2(e) in single precision from one int->float conversion
+// and two lg2.approx.  x < 2^31: w = v below; else 1 - w = v.
+//   w < 2^-6        e = w (1 + w/2)          (series; relative error < w^2/3)
+//   2^-6 <= w < 1/2 e = -ln(1 - w)
+//   w >= 1/2        e = -ln(1 - w), with 1 - w = (~x + 1/2) 2^-32 formed exactly
+// The result is within kScreenCore of log2(e) for every x (host harness and a
+// device test check this over all regimes).
+constexpr float kScreenCore = 1.0f / 2048.0f;
+ERSD_HD float screen_lg2_e(uint32_t x) {
+  const uint32_t t = x ^ (uint32_t)((int32_t)x >> 31);  // x < 2^31 ? x : ~x
+  const float v = fmaf((float)t, 2.3283064365386963e-10f, 1.1641532182693481e-10f);
+  const bool low = (int32_t)x >= 0;
+  const float a = low ? (1.0f - v) : v;
+  const float el = -lg2_fast(a);                           // e / ln 2 (both upper regimes)
+  const float es = v * fmaf(v, 0.5f, 1.0f) * 1.4426950408889634f;  // series, also / ln 2
+  const float e_over_ln2 = (low && v < 0.015625f) ? es : el;
+  return lg2_fast(e_over_ln2) - 0.5287663729448977f;       // + log2(ln 2)
+}
+
+// Slack (log2 units) that makes a comparison of a screening key against a
+// threshold tau safe: |screen key - true key| <= slack(tau) whenever the true
+// key is within a few units of tau.  Covers the core error above, the
+// rounding of log2(e)/T, of the fused multiply-add and of unit conversions.
+ERSD_HD float screen_slack(float tau) { return 0.001953125f + 9.5367431640625e-7f * fabsf(tau); }
+
+}  // namespace ersd

@@ -1,0 +1,382 @@
+"""libersd on the GPU against the CPU oracle, element by element, through the C boundary."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2504_15475_b200 import workloads as wl
+
+from parity_util import KEY_TOL, check_sample, check_verify
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ersd():
+    from paper_2504_15475_b200 import binding
+    binding.lib()
+    assert torch.cuda.is_available()
+    return binding
+
+
+def to_dev(inp):
+    out = dict(inp)
+    for k in ("target", "draft", "seeds", "temps"):
+        if inp.get(k) is not None:
+            out[k] = inp[k].cuda()
+    return out
+
+
+def run_verify(ersd, inp, **kw):
+    d = to_dev(inp)
+    out = ersd.verify(d["target"], d["draft"], d["seeds"], d["T"], temps=d.get("temps"),
+                      parent=d.get("parent"), want_rows=True, **kw)
+    torch.cuda.synchronize()
+    return out
+
+
+# ------------------------------------------------------------------ the five configurations
+def test_config1_tiny_fp32(ersd):
+    inp = wl.make_inputs(wl.CONFIGS["c1"])
+    out = run_verify(ersd, inp)
+    assert check_verify(inp, out) == 0
+    assert out["tokens"].shape == (1, 5)
+
+
+@pytest.mark.parametrize("call", [0, 1, 2, 3])
+def test_config2_calls(ersd, call):
+    inp = wl.make_inputs(wl.CONFIGS["c2"], call=call)
+    out = run_verify(ersd, inp)
+    check_verify(inp, out)
+
+
+@pytest.mark.parametrize("sigma,T", [(0.25, 0.7), (1.0, 1.0), (2.0, 0.7), (2.0, 1.0)])
+def test_config3_points_reduced_batch(ersd, sigma, T):
+    w = wl.scaled(wl.CONFIGS["c3"], B=3)
+    inp = wl.make_inputs(w, sigma=sigma, T=T)
+    out = run_verify(ersd, inp)
+    check_verify(inp, out)
+    acc = out["accept_len"].float().mean().item()
+    assert 0 <= acc <= 8
+
+
+def test_config4_tree_reduced_batch(ersd):
+    w = wl.scaled(wl.CONFIGS["c4"], B=2)
+    inp = wl.make_inputs(w)
+    out = run_verify(ersd, inp)
+    check_verify(inp, out)
+    assert out["tokens"].shape == (2, 5)
+
+
+def test_config5_reduced_batch_per_sequence_temperatures(ersd):
+    w = wl.scaled(wl.CONFIGS["c5"], B=6)
+    inp = wl.make_inputs(w)
+    assert len(set(inp["temps"][:, 0].tolist())) > 1
+    out = run_verify(ersd, inp)
+    check_verify(inp, out)
+
+
+# ------------------------------------------------------------------ full size, sampled sequences
+def _full_size_sampled(ersd, name, sample, **kw):
+    w = wl.CONFIGS[name]
+    inp = wl.make_inputs(w, device="cuda", **kw)
+    out = ersd.verify(inp["target"], inp["draft"], inp["seeds"], inp["T"], temps=inp.get("temps"),
+                      parent=inp.get("parent"), want_rows=True)
+    torch.cuda.synchronize()
+    L = out["accept_len"].cpu().numpy()
+    tok = out["tokens"].cpu().numpy()
+    tt = out["target_tok"].cpu().numpy()
+    B = w.B
+    # properties that hold at any size
+    D = tok.shape[1] - 1
+    assert ((0 <= L) & (L <= D)).all()
+    assert (tt >= 0).all() and (tt < w.V).all()
+    for b in range(B):
+        assert (tok[b, :L[b] + 1] >= 0).all() and (tok[b, L[b] + 1:] == -1).all()
+    if not w.is_tree:
+        dt = out["draft_tok"].cpu().numpy()
+        for b in range(B):
+            assert (tok[b, :L[b] + 1] == tt[b, :L[b] + 1]).all()
+            assert (dt[b, :L[b]] == tt[b, :L[b]]).all()
+            assert L[b] == w.k or dt[b, L[b]] != tt[b, L[b]]
+    # sampled sequences, one by one, against the oracle (sequence id kept)
+    for b in sample:
+        sub = dict(target=inp["target"][b:b + 1], draft=inp["draft"][b:b + 1], seeds=inp["seeds"][b:b + 1],
+                   T=inp["T"], temps=None if inp.get("temps") is None else inp["temps"][b:b + 1],
+                   parent=inp.get("parent"))
+        sub_out = {k: v[b:b + 1] for k, v in out.items()}
+        check_verify(sub, sub_out, seq_ids=[b])
+    return L
+
+
+def test_config3_full_size_sampled(ersd):
+    L = _full_size_sampled(ersd, "c3", sample=(0, 31, 63), sigma=1.0, T=1.0)
+    assert 0.05 < (L > 0).mean() < 1.0
+
+
+def test_config4_full_size_sampled(ersd):
+    _full_size_sampled(ersd, "c4", sample=(0, 31))
+
+
+def test_config5_full_size_sampled(ersd):
+    _full_size_sampled(ersd, "c5", sample=(0, 100, 255))
+
+
+def test_acceptance_tracks_the_closed_form_at_full_vocabulary(ersd):
+    """Config 2 over many calls: the number of accepted first positions falls within 4.5 sigma of
+    the sum of the rows' closed-form match probabilities (computed at full V by sorting on p/q)."""
+    w = wl.CONFIGS["c2"]
+    exp_sum, var_sum, got = 0.0, 0.0, 0
+    for call in range(10, 40):
+        inp = wl.make_inputs(w, call=call)
+        d = to_dev(inp)
+        out = ersd.verify(d["target"], d["draft"], d["seeds"], d["T"])
+        got += int((out["accept_len"] >= 1).sum().item())
+        p = torch.softmax(inp["target"][:, 0].double(), -1).numpy()
+        q = torch.softmax(inp["draft"][:, 0].double(), -1).numpy()
+        for b in range(w.B):
+            r = p[b] / q[b]
+            o = np.argsort(r)
+            ps, qs, rs = p[b][o], q[b][o], r[o]
+            tail_p = np.cumsum(ps[::-1])[::-1]                 # sum of p_j over r_j >= r_i
+            head_q = np.concatenate([[0.0], np.cumsum(qs)[:-1]])  # sum of q_j over r_j < r_i
+            m = float((1.0 / (tail_p / ps + head_q / qs)).sum())
+            exp_sum += m
+            var_sum += m * (1 - m)
+    assert abs(got - exp_sum) < 4.5 * math.sqrt(var_sum), (got, exp_sum)
+
+
+# ------------------------------------------------------------------ edge cases
+@pytest.mark.parametrize("V", [1, 2, 3, 5, 7, 8, 9, 31, 2047, 2048, 2049, 4100, 20000])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_small_and_ragged_vocabularies(ersd, V, dtype):
+    w = wl.Workload("edge", B=3, k=3, V=V, dtype=dtype, sigma=0.7, T=0.9, config_id=40)
+    inp = wl.make_inputs(w, call=V)
+    out = run_verify(ersd, inp)
+    check_verify(inp, out)
+
+
+@pytest.mark.parametrize("split", [1, 2, 3, 7, 32])
+def test_rows_split_over_several_blocks(ersd, split):
+    w = wl.Workload("split", B=2, k=3, V=70001, dtype="bf16", sigma=1.0, T=1.0, config_id=41)
+    inp = wl.make_inputs(w)
+    out = run_verify(ersd, inp, split_v=split)
+    check_verify(inp, out)
+    t = wl.Workload("split_tree", B=2, k=8, V=40000, dtype="bf16", sigma=1.0, T=1.0, config_id=42,
+                    parent=wl.TREE_SPECINFER)
+    inp = wl.make_inputs(t)
+    out = run_verify(ersd, inp, split_v=split)
+    check_verify(inp, out)
+
+
+def test_row_strides_and_unaligned_rows(ersd):
+    B, k, V, ld = 2, 2, 1003, 1011            # odd stride: rows are not 16-byte aligned
+    g = torch.Generator().manual_seed(5)
+    for dtype in (torch.float32, torch.bfloat16):
+        big_t = (torch.randn(B, k + 1, ld, generator=g) * 2).to(dtype)
+        big_d = (torch.randn(B, k, ld, generator=g) * 2).to(dtype)
+        seeds = wl.make_seeds(1, 2, B)
+        opts = ersd.make_opts(ld_target=ld, ld_draft=ld)
+        tok = torch.empty(B, k + 1, dtype=torch.int32, device="cuda")
+        acc = torch.empty(B, dtype=torch.int32, device="cuda")
+        ersd.ersd_verify(big_t.cuda(), big_d.cuda(), seeds.cuda(), 1.0, tok, acc, opts)
+        torch.cuda.synchronize()
+        import oracle
+        ref = oracle.verify(wl.as_numpy_logits(big_t[:, :, :V].contiguous()),
+                            wl.as_numpy_logits(big_d[:, :, :V].contiguous()), wl.seeds_as_u64(seeds), T=1.0)
+        assert (tok.cpu().numpy() == ref["tokens"]).all() and (acc.cpu().numpy() == ref["accept_len"]).all()
+        # base pointer off by one element
+        flat = torch.empty(B * (k + 1) * V + 1, dtype=dtype)
+        flat[1:] = big_t[:, :, :V].reshape(-1)
+        shifted = flat.cuda()[1:].view(B, k + 1, V)
+        drf = big_d[:, :, :V].contiguous().cuda()
+        assert shifted.data_ptr() % 16 != 0
+        ersd.ersd_verify(shifted, drf, seeds.cuda(), 1.0, tok, acc, None)
+        torch.cuda.synchronize()
+        assert (tok.cpu().numpy() == ref["tokens"]).all()
+
+
+def test_special_values(ersd):
+    V = 300
+    g = torch.Generator().manual_seed(9)
+    t = torch.randn(4, 2, V, generator=g)
+    d = torch.randn(4, 1, V, generator=g)
+    t[0, 0, :] = float("-inf")                       # fully masked target row -> -1, nothing accepted
+    t[1, 0, 5] = float("nan")
+    t[1, 0, 100:] = float("-inf")
+    d[1, 0, 17] = float("inf")                       # +inf always wins
+    t[2, 0, :] = float("-inf")
+    t[2, 0, 123] = 0.0                               # single live token
+    d[2, 0, :] = float("nan")
+    d[2, 0, 123] = -3.0
+    for dtype in ("f32", "bf16"):
+        inp = dict(target=wl._storage(t, dtype), draft=wl._storage(d, dtype), seeds=wl.make_seeds(3, 0, 4),
+                   T=0.8, temps=None, parent=None)
+        out = run_verify(ersd, inp)
+        check_verify(inp, out)
+        tok = out["tokens"].cpu().numpy()
+        assert tok[0, 0] == -1 and out["accept_len"][0].item() == 0
+        assert out["draft_tok"][1, 0].item() == 17
+        assert tok[2, 0] == 123 and out["accept_len"][2].item() == 1
+
+
+def test_greedy_temperature_zero(ersd):
+    w = wl.Workload("greedy", B=3, k=2, V=5000, dtype="bf16", sigma=0.3, T=0.0, config_id=43)
+    inp = wl.make_inputs(w)
+    out = run_verify(ersd, inp)
+    check_verify(inp, out)
+    tgt = inp["target"].float()
+    # bf16 rows have many equal maxima candidates: lowest index among the maxima wins
+    am = (tgt == tgt.max(-1, keepdim=True).values).float().argmax(-1)
+    assert (out["target_tok"].cpu() == am).all()
+
+
+def test_per_row_temperatures_sequence_ids_and_offsets(ersd):
+    w = wl.Workload("opts", B=4, k=3, V=3000, dtype="bf16", sigma=0.8, T=1.0, config_id=44)
+    inp = wl.make_inputs(w)
+    temps = torch.tensor([[0.5, 0.7, 1.0, 1.3], [1.0, 1.0, 0.0, 1.0], [2.0, 0.6, 0.6, 0.6], [1.0, -1.0, 1.0, 1.0]])
+    seq = torch.tensor([7, 7, 9, 1000000], dtype=torch.int32)
+    off = torch.tensor([0, 4, 123456, 1], dtype=torch.int32)
+    inp["temps"] = temps
+    out = run_verify(ersd, inp, seq_ids=seq.cuda(), pos_offsets=off.cuda())
+    # the oracle has no notion of an invalid temperature; row (3, 1) must come back as -1
+    assert out["target_tok"][3, 1].item() == -1 and out["draft_tok"][3, 1].item() == -1
+    good = dict(inp)
+    temps_ok = temps.clone()
+    temps_ok[3, 1] = 1.0
+    good["temps"] = temps_ok
+    out_ok = run_verify(ersd, good, seq_ids=seq.cuda(), pos_offsets=off.cuda())
+    check_verify(good, out_ok, seq_ids=seq.numpy().astype(np.uint32), pos_offsets=off.numpy().astype(np.uint32))
+    assert (out["target_tok"][:3].cpu() == out_ok["target_tok"][:3].cpu()).all()
+
+
+def test_no_drafts_and_single_sequence(ersd):
+    w = wl.Workload("k0", B=1, k=0, V=777, dtype="f32", T=1.0, config_id=45)
+    inp = wl.make_inputs(w)
+    d = to_dev(inp)
+    tok = torch.empty(1, 1, dtype=torch.int32, device="cuda")
+    acc = torch.empty(1, dtype=torch.int32, device="cuda")
+    ersd.ersd_verify(d["target"], None, d["seeds"], 1.0, tok, acc, None)
+    torch.cuda.synchronize()
+    import oracle
+    ref_tok, _ = oracle.race_sample(wl.as_numpy_logits(inp["target"]), wl.seeds_as_u64(inp["seeds"]), T=1.0)
+    assert tok.item() == ref_tok.reshape(-1)[0] and acc.item() == 0
+
+
+@pytest.mark.parametrize("parent", [wl.TREE_SPECINFER, wl.star_parent(8), wl.chain_parent(6),
+                                    (-1, 0, 0, 1, 1, 1, 2, 0, 7, 7)])
+def test_tree_shapes(ersd, parent):
+    w = wl.Workload("tree", B=5, k=len(parent) - 1, V=9000, dtype="bf16", sigma=0.6, T=1.0, config_id=46,
+                    parent=tuple(parent))
+    inp = wl.make_inputs(w, call=len(parent))
+    out = run_verify(ersd, inp)
+    check_verify(inp, out)
+
+
+def test_wide_star_uses_many_arrivals(ersd):
+    parent = wl.star_parent(32)
+    w = wl.Workload("star32", B=3, k=32, V=5000, dtype="f32", sigma=0.5, T=1.0, config_id=47,
+                    parent=tuple(parent))
+    inp = wl.make_inputs(w)
+    out = run_verify(ersd, inp)
+    check_verify(inp, out)
+    dt = out["draft_tok"][:, 1:].cpu().numpy()
+    assert all(len(set(r.tolist())) == 32 for r in dt)
+
+
+# ------------------------------------------------------------------ race sampling
+@pytest.mark.parametrize("c,split", [(1, 0), (1, 3), (4, 0), (4, 2), (32, 0), (32, 2)])
+def test_race_sample_first_arrivals(ersd, c, split):
+    B, R, V = 3, 4, 33000
+    g = torch.Generator().manual_seed(c)
+    logits = wl.zipf_rows(B * R, V, g, "cpu").view(B, R, V).to(torch.bfloat16)
+    seeds = wl.make_seeds(11, c, B)
+    tok = torch.empty(B, R, c, dtype=torch.int32, device="cuda")
+    key = torch.empty(B, R, c, dtype=torch.float32, device="cuda")
+    ersd.ersd_race_sample(logits.cuda(), seeds.cuda(), 0.9, tok, ersd.make_opts(top_c=c, split_v=split, out_key=key))
+    torch.cuda.synchronize()
+    check_sample(logits, seeds, 0.9, tok, key, c=c)
+
+
+def test_race_sample_draft_then_verify_is_consistent(ersd):
+    """Drafting with race_sample and verifying with ersd_verify see the same draft winners."""
+    w = wl.scaled(wl.CONFIGS["c2"], B=4)
+    inp = to_dev(wl.make_inputs(w, call=77))
+    tok = torch.empty(w.B, w.k, 1, dtype=torch.int32, device="cuda")
+    ersd.ersd_race_sample(inp["draft"], inp["seeds"], inp["T"], tok, None)
+    out = ersd.verify(inp["target"], inp["draft"], inp["seeds"], inp["T"], want_rows=True)
+    torch.cuda.synchronize()
+    assert (tok[..., 0] == out["draft_tok"]).all()
+
+
+# ------------------------------------------------------------------ keys, workspace, repeats
+def test_row_keys_match_the_oracle(ersd):
+    import oracle
+    V = 50000
+    g = torch.Generator().manual_seed(3)
+    row = wl.zipf_rows(1, V, g, "cpu")[0].to(torch.bfloat16)
+    out0 = torch.empty(V, dtype=torch.float32, device="cuda")
+    out1 = torch.empty(V, dtype=torch.float32, device="cuda")
+    seed = 0x1234567890ABCDEF
+    for T in (0.6, 1.0):
+        ersd.ersd_row_keys(row.cuda(), T, seed, 3, 9, 0, out0)
+        ersd.ersd_row_keys(row.cuda(), T, seed, 3, 9, 1, out1)
+        torch.cuda.synchronize()
+        ref = oracle.row_keys(wl.as_numpy_logits(row), float(np.float32(T)), seed, 3, 9)
+        e0 = np.abs(out0.cpu().numpy().astype(np.float64) - ref)
+        assert e0.max() <= KEY_TOL, e0.max()
+        # screening keys on the device (lg2.approx): within half the slack the kernel allows
+        e1 = np.abs(out1.cpu().numpy().astype(np.float64) - ref) / math.log(2)
+        slack = 2.0**-9 + 2.0**-20 * np.abs(ref) / math.log(2)
+        assert (e1 <= 0.5 * slack).all(), (e1 / slack).max()
+
+
+def test_screening_log_on_the_device_over_all_regimes(ersd):
+    """Zero logits, T = 1: key = ln e.  Sweeps small, switch-point and large x through real lg2.approx."""
+    import oracle
+    V = 1 << 20
+    row = torch.zeros(V, dtype=torch.float32, device="cuda")
+    out1 = torch.empty(V, dtype=torch.float32, device="cuda")
+    worst = 0.0
+    for pos in range(4):
+        ersd.ersd_row_keys(row, 1.0, 42, 0, pos, 1, out1)
+        torch.cuda.synchronize()
+        ref = oracle.row_keys(np.zeros(V, np.float32), 1.0, 42, 0, pos)
+        worst = max(worst, float(np.abs(out1.cpu().numpy() - ref).max()) / math.log(2))
+    assert worst < 2.0**-11
+
+
+def test_caller_owned_workspace_and_repeats(ersd):
+    w = wl.scaled(wl.CONFIGS["c2"], B=3)
+    inp = to_dev(wl.make_inputs(w, call=5))
+    nbytes = ersd.ersd_workspace_bytes(w.B, w.k + 1)
+    guard = 64
+    buf = torch.full((nbytes + 2 * guard,), 0x5A, dtype=torch.uint8, device="cuda")
+    ws = buf[guard:guard + nbytes]
+    ersd.ersd_workspace_init(ws)
+    first = None
+    for rep in range(30):
+        tok = torch.full((w.B, w.k + 1), -7, dtype=torch.int32, device="cuda")
+        acc = torch.full((w.B,), -7, dtype=torch.int32, device="cuda")
+        ersd.ersd_verify(inp["target"], inp["draft"], inp["seeds"], 1.0, tok, acc,
+                         ersd.make_opts(workspace=ws, split_v=1 + rep % 4))
+        torch.cuda.synchronize()
+        if first is None:
+            first = (tok.clone(), acc.clone())
+        assert (tok == first[0]).all() and (acc == first[1]).all()
+    assert (buf[:guard] == 0x5A).all() and (buf[guard + nbytes:] == 0x5A).all()   # canaries intact
+    small = ersd.make_opts(workspace=ws[:64])
+    with pytest.raises(ersd.ErsdError) as e:
+        ersd.ersd_verify(inp["target"], inp["draft"], inp["seeds"], 1.0, tok, acc, small)
+    assert e.value.status == -5
+
+
+def test_host_buffer_entry(ersd):
+    w = wl.scaled(wl.CONFIGS["c2"], B=2)
+    inp = wl.make_inputs(w, call=8)
+    tok, acc = ersd.verify_host(inp["target"].pin_memory(), inp["draft"].pin_memory(), inp["seeds"], inp["T"])
+    import oracle
+    ref = oracle.verify(wl.as_numpy_logits(inp["target"]), wl.as_numpy_logits(inp["draft"]),
+                        wl.seeds_as_u64(inp["seeds"]), T=inp["T"])
+    assert (acc.numpy() == ref["accept_len"]).all()
