@@ -42,7 +42,8 @@
  *   - Scratch memory: calls that split rows over several thread blocks, and
  *     every verify call, exchange partial results through a workspace.  Give
  *     one in opts->workspace (size from ersd_workspace_bytes, zeroed once
- *     with ersd_workspace_init; the library leaves it zeroed) or pass none
+ *     with ersd_workspace_init; every call leaves it ready for the next
+ *     call, of any size that fits) or pass none
  *     and the library keeps a private one per device, (re)allocated with
  *     cudaMalloc when a call needs more than it holds.  Two calls that may
  *     overlap on the GPU must not share a workspace.

@@ -34,6 +34,15 @@ struct Entry {  // one arrival: race key (natural-log units) and token id
   int32_t pad;
 };
 
+// Workspace layout: one slot per logit row, whatever the call's sizes, so that a counter field
+// is never reused as a partial-list field by a later call with other sizes (counters must be
+// zero when a call starts; partial lists are always rewritten before they are read).
+struct Slot {
+  int counter;  // arrivals of the group whose first row this is; reset to 0 by the last arrival
+  int pad[3];
+  Entry part[2][kPartCap];  // per role: S partial lists of c entries each
+};
+
 struct TreeDesc {  // draft tree of one call, passed by value in kernel parameter space
   int16_t parent[ERSD_MAX_ROWS];
   int16_t first_child[ERSD_MAX_ROWS];
@@ -71,8 +80,7 @@ struct Params {
   int32_t* out_target_tok;
   float* out_target_key;
   float* out_key;        // sample mode
-  int* counters;
-  Entry* partials;
+  Slot* slots;
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -385,7 +393,7 @@ ersd_race_kernel(const Params p, const __grid_constant__ TreeDesc tree) {
       e.key = L.key;
       e.idx = L.idx;
       e.pad = 0;
-      p.partials[((size_t)unit * 2 + role) * kPartCap + (size_t)s * c + lane] = e;
+      p.slots[unit].part[role][s * c + lane] = e;
     }
   }
   if (direct) return;
@@ -393,21 +401,21 @@ ersd_race_kernel(const Params p, const __grid_constant__ TreeDesc tree) {
   // ---- the last block of the group (row in sample mode, sequence otherwise) finishes ----
   __threadfence();
   __syncthreads();
-  const int group = (p.mode == kSample) ? unit : b;
+  int* counter = &p.slots[(p.mode == kSample) ? unit : b * p.rows].counter;
   const int group_items = (p.mode == kSample) ? p.S : p.rows * p.S;
   if (tid == 0) {
-    const int old = atomicAdd(&p.counters[group], 1);
+    const int old = atomicAdd(counter, 1);
     sm_last = (old == group_items - 1);
   }
   __syncthreads();
   if (!sm_last) return;
   __threadfence();
-  if (tid == 0) p.counters[group] = 0;  // leave the workspace zeroed for the next call
+  if (tid == 0) *counter = 0;  // leave the workspace ready for the next call
 
   if (p.mode == kSample) {
     if (warp == 0) {
       WarpList L;
-      merge_partials(L, p.partials + (size_t)unit * 2 * kPartCap, p.S, c0, lane);
+      merge_partials(L, p.slots[unit].part[0], p.S, c0, lane);
       if (lane < c0) {
         const bool ok = L.idx != 0x7FFFFFFF;
         const size_t o = (size_t)unit * c0 + lane;
@@ -424,7 +432,7 @@ ersd_race_kernel(const Params p, const __grid_constant__ TreeDesc tree) {
     const int c = role ? (int)tree.nchild[n] : 1;
     if (c == 0) continue;
     WarpList L;
-    merge_partials(L, p.partials + ((size_t)(b * p.rows + n) * 2 + role) * kPartCap, p.S, c, lane);
+    merge_partials(L, p.slots[b * p.rows + n].part[role], p.S, c, lane);
     const bool ok = L.idx != 0x7FFFFFFF;
     if (role == 0) {
       if (lane == 0) {
@@ -528,8 +536,7 @@ static OwnedWorkspace g_ws[64];
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 static size_t workspace_bytes(int64_t B, int64_t rows) {
-  const size_t units = (size_t)B * (size_t)rows;
-  return align_up(units * sizeof(int), 256) + units * 2 * kPartCap * sizeof(Entry);
+  return (size_t)B * (size_t)rows * sizeof(Slot);
 }
 
 static int get_workspace(const ersd_opts& o, size_t need, void** ws) {
@@ -715,8 +722,7 @@ static int verify_impl(const void* target, const void* draft, int dt, const Tree
   void* ws = nullptr;
   const int st = get_workspace(o, workspace_bytes(B, rows), &ws);
   if (st != ERSD_OK) return st;
-  p.counters = (int*)ws;
-  p.partials = (Entry*)((char*)ws + align_up((size_t)B * rows * sizeof(int), 256));
+  p.slots = (Slot*)ws;
   return launch(p, tree, dt, (cudaStream_t)stream);
 }
 
@@ -752,8 +758,7 @@ int ersd_race_sample(const void* logits, ersd_dtype dt, const uint64_t* seeds, i
     void* ws = nullptr;
     st = get_workspace(o, workspace_bytes(B, R), &ws);
     if (st != ERSD_OK) return st;
-    p.counters = (int*)ws;
-    p.partials = (Entry*)((char*)ws + align_up((size_t)B * R * sizeof(int), 256));
+    p.slots = (Slot*)ws;
   }
   TreeDesc tree;
   memset(&tree, 0, sizeof tree);

@@ -372,6 +372,34 @@ def test_caller_owned_workspace_and_repeats(ersd):
     assert e.value.status == -5
 
 
+def test_workspace_reused_by_calls_of_different_sizes(ersd):
+    """A small call leaves partial lists behind; a larger call on the same workspace must not
+    mistake them for arrival counters (and the other way round)."""
+    shapes = [(2, 1, 9000), (40, 4, 3000), (3, 7, 20000), (64, 2, 2500), (1, 0, 5000)]
+    nbytes = max(ersd.ersd_workspace_bytes(B, k + 1) for B, k, _ in shapes)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    ersd.ersd_workspace_init(ws)
+    for rnd in range(2):
+        for n, (B, k, V) in enumerate(shapes):
+            w = wl.Workload("ws", B=B, k=k, V=V, dtype="bf16", sigma=0.8, T=1.0, config_id=48)
+            inp = wl.make_inputs(w, call=n)
+            d = to_dev(inp)
+            tok = torch.empty(B, k + 1, dtype=torch.int32, device="cuda")
+            acc = torch.empty(B, dtype=torch.int32, device="cuda")
+            ersd.ersd_verify(d["target"], d["draft"] if k else None, d["seeds"], 1.0, tok, acc,
+                             ersd.make_opts(workspace=ws, split_v=(0, 2)[rnd]))
+            torch.cuda.synchronize()
+            import oracle
+            if k:
+                ref = oracle.verify(wl.as_numpy_logits(inp["target"]), wl.as_numpy_logits(inp["draft"]),
+                                    wl.seeds_as_u64(inp["seeds"]), T=1.0)
+                if min((ref["target_key"][..., 1] - ref["target_key"][..., 0]).min(),
+                       (ref["draft_key"][..., 1] - ref["draft_key"][..., 0]).min()) < 1e-5:
+                    continue
+                assert (tok.cpu().numpy() == ref["tokens"]).all(), (rnd, n)
+                assert (acc.cpu().numpy() == ref["accept_len"]).all(), (rnd, n)
+
+
 def test_host_buffer_entry(ersd):
     w = wl.scaled(wl.CONFIGS["c2"], B=2)
     inp = wl.make_inputs(w, call=8)
