@@ -70,12 +70,14 @@ typedef enum {
   ERSD_EALIGN = -2,       /* pointer not aligned to its element size */
   ERSD_EUNSUPPORTED = -3, /* size beyond a compiled limit (see ERSD_MAX_*) */
   ERSD_ECUDA = -4,        /* a CUDA runtime call failed; see ersd_last_cuda_error() */
-  ERSD_EWORKSPACE = -5    /* opts->workspace given but too small */
+  ERSD_EWORKSPACE = -5,   /* opts->workspace given but too small */
+  ERSD_ENOALLOC_LIMIT = -6 /* ersd_verify_noalloc: B * (k + 1) > ERSD_NOALLOC_MAX_ROWS */
 } ersd_status;
 
 #define ERSD_MAX_TOP_C 32   /* arrivals per race (children per tree node, opts->top_c) */
 #define ERSD_MAX_ROWS 256   /* rows per sequence: k + 1, N + 1 */
 #define ERSD_MAX_SPLIT 32   /* thread blocks sharing one row */
+#define ERSD_NOALLOC_MAX_ROWS 1024 /* ersd_verify_noalloc: largest B * (k + 1) */
 
 /* Optional arguments.  Pass NULL for defaults.  Set struct_size = sizeof(ersd_opts). */
 typedef struct ersd_opts {
@@ -157,6 +159,42 @@ int ersd_verify_tree(const void* target_logits, const void* draft_logits, ersd_d
                      const int32_t* parent, const uint64_t* seeds, int B, int N, int V, float T,
                      int32_t* out_tokens, int32_t* out_accept_len, const ersd_opts* opts,
                      void* cuda_stream);
+
+/*
+ * ersd_verify for callers that must not allocate device memory.  (The paper has
+ * no counterpart; this is a deployment variant of ersd_verify and computes
+ * exactly the same outputs from the same arguments.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a
+ * serving loop whose memory is fully pre-planned by a pool allocator, in a
+ * latency-critical section where the implicit device synchronisation of
+ * cudaMalloc/cudaFree is unacceptable, or in a process whose device memory is
+ * already handed out to the last byte.  ersd_verify either wants a workspace
+ * from the caller or grows a private one with cudaMalloc; this entry point does
+ * neither.  Its scratch is a fixed array of about 2.1 MB compiled into the
+ * library image (every GPU that loads the library holds that much until the
+ * process exits), sized for B * (k + 1) <= ERSD_NOALLOC_MAX_ROWS.  Larger calls
+ * are refused with ERSD_ENOALLOC_LIMIT and nothing is launched.  The call makes
+ * no cudaMalloc, cudaFree or other allocating call.
+ *
+ * Arguments, outputs and errors are those of ersd_verify, except that
+ * opts->workspace must be NULL (ERSD_EINVAL otherwise).
+ *
+ * First call on a device: the library looks up the array's device address
+ * (once per device, with the caller's current device) before it launches.
+ * Make that first call outside any stream capture; a throw-away call at
+ * start-up is enough.
+ *
+ * Sharing: every call on a device uses the same array, which still holds what
+ * the previous call left there.  The library clears the part that must start
+ * at zero on `cuda_stream` before each launch.  Two calls that can overlap on
+ * the GPU (different streams, or different host threads without ordering
+ * between them) race on the array and give wrong results; serialise them, or
+ * use ersd_verify with one workspace per stream.
+ */
+int ersd_verify_noalloc(const void* target_logits, const void* draft_logits, ersd_dtype dt,
+                        const uint64_t* seeds, int B, int k, int V, float T, int32_t* out_tokens,
+                        int32_t* out_accept_len, const ersd_opts* opts, void* cuda_stream);
 
 /* Depth (longest root-to-leaf edge count) of a HOST parent array, or -1 if it is malformed. */
 int ersd_tree_depth(const int32_t* parent, int N);

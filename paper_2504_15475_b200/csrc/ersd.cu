@@ -726,6 +726,34 @@ static int verify_impl(const void* target, const void* draft, int dt, const Tree
   return launch(p, tree, dt, (cudaStream_t)stream);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Scratch for ersd_verify_noalloc: lives in the library image, one copy per GPU that loads it.
+// In host code `g_noalloc_scratch` is only a handle for the runtime, never an address to hand
+// to a kernel; noalloc_scratch() asks the runtime for the device address, once per device.
+// ---------------------------------------------------------------------------------------------
+constexpr size_t kNoallocBytes = (size_t)ERSD_NOALLOC_MAX_ROWS * sizeof(Slot);
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoallocBytes];
+
+static std::mutex g_noalloc_mutex;
+static void* g_noalloc_ptr[64];
+
+static int noalloc_scratch(void** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (dev < 0 || dev >= 64) return ERSD_EUNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  if (!g_noalloc_ptr[dev]) {
+    void* ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);  // address on the current device
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (!ptr) return ERSD_ECUDA;
+    g_noalloc_ptr[dev] = ptr;
+  }
+  *out = g_noalloc_ptr[dev];
+  return ERSD_OK;
+}
+
 }  // namespace ersd
 
 using namespace ersd;
@@ -808,6 +836,28 @@ int ersd_verify_tree(const void* target_logits, const void* draft_logits, ersd_d
                      V, T, out_tokens, out_accept_len, opts, cuda_stream);
 }
 
+int ersd_verify_noalloc(const void* target_logits, const void* draft_logits, ersd_dtype dt,
+                        const uint64_t* seeds, int B, int k, int V, float T, int32_t* out_tokens,
+                        int32_t* out_accept_len, const ersd_opts* opts, void* cuda_stream) {
+  if (B < 1 || k < 0) return ERSD_EINVAL;
+  if ((int64_t)B * ((int64_t)k + 1) > ERSD_NOALLOC_MAX_ROWS) return ERSD_ENOALLOC_LIMIT;
+  ersd_opts o = read_opts(opts);
+  if (o.workspace) return ERSD_EINVAL;  // this entry point brings its own scratch
+  void* scratch = nullptr;
+  const int st = noalloc_scratch(&scratch);
+  if (st != ERSD_OK) return st;
+  // The array keeps whatever the previous call left; the arrival counters (the first 16 bytes
+  // of every slot this call uses) must start at zero.
+  const cudaError_t e = cudaMemset2DAsync(scratch, sizeof(Slot), 0, 16, (size_t)B * ((size_t)k + 1),
+                                          (cudaStream_t)cuda_stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  o.struct_size = sizeof o;
+  o.workspace = scratch;
+  o.workspace_bytes = kNoallocBytes;
+  return ersd_verify(target_logits, draft_logits, dt, seeds, B, k, V, T, out_tokens, out_accept_len,
+                     &o, cuda_stream);
+}
+
 int ersd_tree_depth(const int32_t* parent, int N) {
   if (!parent || N < 0 || N + 1 > ERSD_MAX_ROWS) return -1;
   TreeDesc tree;
@@ -851,6 +901,8 @@ const char* ersd_status_string(int status) {
     case ERSD_EUNSUPPORTED: return "size beyond a compiled limit";
     case ERSD_ECUDA: return "CUDA runtime error";
     case ERSD_EWORKSPACE: return "workspace too small";
+    case ERSD_ENOALLOC_LIMIT:
+      return "B * (k + 1) exceeds ERSD_NOALLOC_MAX_ROWS, the capacity of ersd_verify_noalloc's built-in scratch";
     default: return "unknown status";
   }
 }
