@@ -214,10 +214,45 @@ struct Role {
   WarpList list;
 };
 
-// Screen eight indices of one role and, where needed, evaluate exactly and insert.
+// Shared-memory float minimum (rare path).
+__device__ __forceinline__ void smem_min(float* addr, float v) {
+  float old = *(volatile float*)addr;
+  while (v < old) {
+    const float seen = __int_as_float(atomicCAS((int*)addr, __float_as_int(old), __float_as_int(v)));
+    if (seen == old) break;
+    old = seen;
+  }
+}
+
+// Upper bound of the eight logits of a tile slice (NaN ignored; NaN if all are NaN).
+__device__ __forceinline__ float logits_upper_bound(const Raw<ERSD_BF16>& r) {
+  uint32_t m01, m23, m;
+  asm("max.bf16x2 %0, %1, %2;" : "=r"(m01) : "r"(r.a.x), "r"(r.a.y));
+  asm("max.bf16x2 %0, %1, %2;" : "=r"(m23) : "r"(r.a.z), "r"(r.a.w));
+  asm("max.bf16x2 %0, %1, %2;" : "=r"(m) : "r"(m01), "r"(m23));
+  // The odd elements' maximum sits in the high half.  Read with the low half attached it is
+  // off by less than one bf16 ulp (2^-7 relative, towards larger magnitude); widen it to a
+  // sure upper bound instead of masking.
+  const float hi_raw = __uint_as_float(m);
+  const float hi_ub = fmaf(fabsf(hi_raw), 0.0078125f, hi_raw);
+  const float lo = __uint_as_float(m << 16);
+  return fmaxf(hi_ub, lo);
+}
+__device__ __forceinline__ float logits_upper_bound(const Raw<ERSD_F32>& r) {
+  const float a = fmaxf(fmaxf(__uint_as_float(r.a.x), __uint_as_float(r.a.y)),
+                        fmaxf(__uint_as_float(r.a.z), __uint_as_float(r.a.w)));
+  const float b = fmaxf(fmaxf(__uint_as_float(r.b.x), __uint_as_float(r.b.y)),
+                        fmaxf(__uint_as_float(r.b.z), __uint_as_float(r.b.w)));
+  return fmaxf(a, b);
+}
+
+// Examine eight indices of one role: a[j] = lg[j] - z[j] * c2 is either the screening key
+// (`accurate`: within the slack of the true key, so the c-th smallest lane minimum also
+// tightens tau) or only a lower bound of it.  Indices that can still be among the first c
+// arrivals are evaluated in double precision and inserted into the warp's list.
 __device__ __forceinline__ void race_role(Role& R, const float z[8], const float lg[8],
                                           const uint32_t xs[8], int i0, float c2, float T,
-                                          int* sm_tau, int lane) {
+                                          float* sm_tau, int lane, bool accurate) {
   float a[8];
   float m = INFINITY;
 #pragma unroll
@@ -225,11 +260,14 @@ __device__ __forceinline__ void race_role(Role& R, const float z[8], const float
     a[j] = fmaf(-z[j], c2, lg[j]);
     m = fminf(m, a[j]);
   }
-  float tau = fminf(R.tau, float_of(*(volatile int*)sm_tau));
+  const float tau_in = fminf(R.tau, *(volatile float*)sm_tau);
+  float tau = tau_in;
   const bool hit = m <= tau + screen_slack(tau);
   if (__any_sync(kFull, hit)) {
-    const float theta = cth_smallest(m, R.c, lane);
-    tau = fminf(tau, theta + screen_slack(theta));
+    if (accurate) {
+      const float theta = cth_smallest(m, R.c, lane);
+      tau = fminf(tau, theta + screen_slack(theta));
+    }
     const float lim = tau + screen_slack(tau);
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
@@ -249,15 +287,22 @@ __device__ __forceinline__ void race_role(Role& R, const float z[8], const float
     }
     const double kc = R.list.key_at(R.c - 1);
     if (kc < (double)INFINITY) tau = fminf(tau, tau_of_exact(kc));
-    if (lane == 0 && tau < INFINITY) atomicMin(sm_tau, ord_of(tau));
+    if (lane == 0 && tau < tau_in) smem_min(sm_tau, tau);
   }
   R.tau = tau;
 }
 
+// Stream one chunk [v0, v1) of a row (NR = 1) or of a draft/target pair (NR = 2).
+//
+// Fast path per thread and tile of eight indices: two Philox calls, the smallest of the eight
+// words, the largest of the eight logits per role, and one comparison per role of
+//     lg2(x_min) - z_max * c2      (a lower bound of all eight keys, shifted by 32)
+// against the block's threshold.  Only when some lane of the warp cannot rule its eight
+// indices out does the warp look at them one by one (race_role).
 template <int DT, int NR>
-__device__ __forceinline__ void stream_chunk(Role* roles, int v0, int v1, uint32_t k0,
-                                             uint32_t k1, uint32_t pos, uint32_t seq, float c2,
-                                             float T, bool greedy, int* sm_tau, int lane) {
+__device__ __forceinline__ void stream_chunk(Role* roles, int v0, int v1, const PhiloxRow& pr,
+                                             float c2, float T, bool greedy, float* sm_tau,
+                                             int lane) {
   const int tid = threadIdx.x;
   const int ntiles = (v1 - v0 + kTile - 1) / kTile;
   Raw<DT> cur[NR], nxt[NR];
@@ -271,16 +316,34 @@ __device__ __forceinline__ void stream_chunk(Role* roles, int v0, int v1, uint32
       for (int r = 0; r < NR; ++r) nxt[r] = fetch<DT>(roles[r].row, in, v1, roles[r].aligned);
     }
     uint32_t xs[8];
-    float lg[8];
-    philox4x32_10((uint32_t)i0 >> 2, pos, seq, 0u, k0, k1, xs);
-    philox4x32_10(((uint32_t)i0 >> 2) + 1u, pos, seq, 0u, k0, k1, xs + 4);
-#pragma unroll
-    for (int j = 0; j < 8; ++j) lg[j] = greedy ? 0.0f : screen_lg2_e(xs[j]);
+    pr.words((uint32_t)i0 >> 2, xs);
+    pr.words(((uint32_t)i0 >> 2) + 1u, xs + 4);
+    const uint32_t xm = min(min(min(xs[0], xs[1]), min(xs[2], xs[3])),
+                            min(min(xs[4], xs[5]), min(xs[6], xs[7])));
+    // lg2(w) >= lg2(x) - 32; the 32 moves to the threshold's side.  Greedy rows have no race.
+    const float lgm = greedy ? 32.0f : lg2_fast((float)xm);
+    bool pass = false, boot = false;
 #pragma unroll
     for (int r = 0; r < NR; ++r) {
-      float z[8];
-      decode(cur[r], z);
-      race_role(roles[r], z, lg, xs, i0, c2, T, sm_tau + r, lane);
+      const float tau = *(volatile float*)(sm_tau + r);
+      const float lim32 = fmaf(fabsf(tau), 9.5367431640625e-7f, tau) + 32.001953125f;
+      const float lb = fmaf(-logits_upper_bound(cur[r]), c2, lgm);
+      pass |= !(lb > lim32);
+      boot |= !(tau < INFINITY);
+    }
+    if (__any_sync(kFull, pass)) {
+      // No threshold yet (first tiles of a chunk): use the accurate screening value so that
+      // the tile itself yields one.  Otherwise the cheaper lower bound lg2(x) - 32 will do.
+      float lg[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        lg[j] = greedy ? 0.0f : (boot ? screen_lg2_e(xs[j]) : lg2_fast((float)xs[j]) - 32.0f);
+#pragma unroll
+      for (int r = 0; r < NR; ++r) {
+        float z[8];
+        decode(cur[r], z);
+        race_role(roles[r], z, lg, xs, i0, c2, T, sm_tau + r, lane, boot || greedy);
+      }
     }
 #pragma unroll
     for (int r = 0; r < NR; ++r) cur[r] = nxt[r];
@@ -300,10 +363,14 @@ __device__ __forceinline__ void merge_partials(WarpList& L, const Entry* part, i
   }
 }
 
+#ifndef ERSD_MIN_BLOCKS
+#define ERSD_MIN_BLOCKS 2  // resident blocks per SM the register allocation aims for
+#endif
+
 template <int DT>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, ERSD_MIN_BLOCKS)
 ersd_race_kernel(const Params p, const __grid_constant__ TreeDesc tree) {
-  __shared__ int sm_tau[2];
+  __shared__ float sm_tau[2];
   __shared__ Entry sm_list[2][kWarps][ERSD_MAX_TOP_C];
   __shared__ int sm_last;
   __shared__ int sm_ttok[ERSD_MAX_ROWS], sm_dtok[ERSD_MAX_ROWS];
@@ -335,8 +402,10 @@ ersd_race_kernel(const Params p, const __grid_constant__ TreeDesc tree) {
   else if (T > 0.0f && T < INFINITY) c2 = (float)(1.4426950408889634 / (double)T);
   else c2 = __int_as_float(0x7FC00000);  // invalid temperature: no token arrives
 
-  if (tid < 2) sm_tau[tid] = ord_of(INFINITY);
+  if (tid < 2) sm_tau[tid] = INFINITY;
   __syncthreads();
+  PhiloxRow pr;
+  pr.init(seed, seq, pos);
 
   const size_t es = (DT == ERSD_BF16) ? 2 : 4;
   Role roles[2];
@@ -352,16 +421,16 @@ ersd_race_kernel(const Params p, const __grid_constant__ TreeDesc tree) {
   roles[1].list.init();
   if (cq > 0) {
     roles[1].row = (const char*)p.draft + ((size_t)b * p.draft_rows + r) * (size_t)p.ld_d * es;
-    stream_chunk<DT, 2>(roles, v0, v1, (uint32_t)seed, (uint32_t)(seed >> 32), pos, seq, c2, T,
-                        greedy, sm_tau, lane);
+    stream_chunk<DT, 2>(roles, v0, v1, pr, c2, T, greedy, sm_tau, lane);
   } else {
-    stream_chunk<DT, 1>(roles, v0, v1, (uint32_t)seed, (uint32_t)(seed >> 32), pos, seq, c2, T,
-                        greedy, sm_tau, lane);
+    stream_chunk<DT, 1>(roles, v0, v1, pr, c2, T, greedy, sm_tau, lane);
   }
 
   // ---- block merge: every warp publishes its list, warp `role` merges that role's lists ----
   const int nroles = cq > 0 ? 2 : 1;
-  for (int role = 0; role < nroles; ++role) {
+#pragma unroll
+  for (int role = 0; role < 2; ++role) {
+    if (role >= nroles) break;
     Entry e;
     e.key = roles[role].list.key;
     e.idx = roles[role].list.idx;
@@ -372,8 +441,8 @@ ersd_race_kernel(const Params p, const __grid_constant__ TreeDesc tree) {
   const bool direct = (p.mode == kSample && p.S == 1);
   if (warp < nroles) {
     const int role = warp;
-    const int c = roles[role].c;
-    WarpList L = roles[role].list;
+    const int c = role ? roles[1].c : roles[0].c;
+    WarpList L = role ? roles[1].list : roles[0].list;
     for (int w = 0; w < kWarps; ++w) {
       if (w == warp) continue;
       for (int e = 0; e < c; ++e) {

@@ -9,6 +9,11 @@ void ersd_host_philox(const uint32_t* ctr, const uint32_t* key, uint32_t* out) {
 uint32_t ersd_host_token_word(uint64_t seed, uint32_t seq, uint32_t pos, uint32_t i) {
   return ersd::token_word(seed, seq, pos, i);
 }
+void ersd_host_philox_row(uint64_t seed, uint32_t seq, uint32_t pos, uint32_t c0, uint32_t* out) {
+  ersd::PhiloxRow pr;
+  pr.init(seed, seq, pos);
+  pr.words(c0, out);
+}
 double ersd_host_exact_ln_e(uint32_t x) { return ersd::exact_ln_e(x); }
 double ersd_host_exact_key(uint32_t x, float z, float T) { return ersd::exact_key(x, z, T); }
 float ersd_host_screen_lg2_e(uint32_t x) { return ersd::screen_lg2_e(x); }

@@ -60,6 +60,23 @@ def test_library_philox_matches_published_vectors(hm):
         assert hm.ersd_host_token_word(seed, 22, 11, i) == out[i & 3]
 
 
+def test_row_folded_philox_equals_the_plain_one(hm):
+    rng = np.random.default_rng(3)
+    hm.ersd_host_philox_row.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, C.c_void_p]
+    for _ in range(300):
+        seed = int(rng.integers(0, 2**63)) * 2 + int(rng.integers(0, 2))
+        seq, pos, c0 = (int(v) for v in rng.integers(0, 2**32, size=3))
+        if _ % 7 == 0:
+            seq, pos = 0, 0
+        ctr = (C.c_uint32 * 4)(c0, pos, seq, 0)
+        key = (C.c_uint32 * 2)(seed & 0xFFFFFFFF, seed >> 32)
+        a = (C.c_uint32 * 4)()
+        b = (C.c_uint32 * 4)()
+        hm.ersd_host_philox(ctr, key, a)
+        hm.ersd_host_philox_row(seed, seq, pos, c0, b)
+        assert list(a) == list(b)
+
+
 def _xs():
     rng = np.random.default_rng(0)
     edges = [0, 1, 2, 3, 255, 256, 2**16, 2**23 - 1, 2**23, 2**23 + 1, 2**24, 2**24 + 1,
