@@ -1,12 +1,14 @@
 // libersd: exponential-race speculative decoding kernels for sm_100a and their C entry points.
 //
 // One thread block streams one chunk of one logit row (or of a draft/target
-// row pair that shares its race variables).  Per vocabulary index it draws the
-// 32-bit Philox word, forms a cheap single-precision screening key and keeps
-// only the indices that can still be among the first c arrivals; those few
-// are re-evaluated in double precision and inserted into a per-warp sorted
-// list.  Lists are merged per block, exchanged through a small workspace, and
-// the last block of a sequence turns the winners into the accepted prefix
+// row pair that shares its race variables).  Logits arrive through a
+// shared-memory ring filled by cp.async; per group of eight vocabulary indices
+// a thread draws the Philox words and compares one cheap lower bound of the
+// eight race keys with the block's running threshold.  The few groups that
+// survive are screened index by index in single precision and the survivors of
+// that are decided in double precision and kept in per-warp sorted lists.
+// Lists are merged per block, exchanged through a small workspace, and the
+// last block of a sequence turns the winners into the accepted prefix
 // (sequence scan or tree walk) in the same launch.
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -100,15 +102,32 @@ __device__ __forceinline__ uint4 ldg_stream(const void* p) {
   return v;
 }
 
+// 16-byte asynchronous copy global -> shared (bypasses L1); completion is tracked per thread.
+__device__ __forceinline__ void cp_async16(uint32_t smem_addr, const void* gptr) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr), "l"(gptr) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+// Geometry per logit type: a thread owns eight consecutive logits of a tile, i.e. kVec 16-byte
+// vectors per role; the shared-memory ring holds kStages tiles per role (32 KB either way).
 template <int DT>
-struct Raw;
+struct Geo;
 template <>
-struct Raw<ERSD_BF16> {
-  uint4 a;
+struct Geo<ERSD_BF16> {
+  static constexpr int kVec = 1, kStages = 4;
 };
 template <>
-struct Raw<ERSD_F32> {
-  uint4 a, b;
+struct Geo<ERSD_F32> {
+  static constexpr int kVec = 2, kStages = 2;
+};
+
+template <int DT>
+struct Raw {
+  uint4 v[Geo<DT>::kVec];
 };
 
 // Eight logits starting at element i0 of a row; elements at or beyond `vend` read as NaN.
@@ -118,7 +137,7 @@ __device__ __forceinline__ Raw<DT> fetch(const void* row, int i0, int vend, bool
   if constexpr (DT == ERSD_BF16) {
     const uint16_t* p = (const uint16_t*)row;
     if (aligned && i0 + kPerThread <= vend) {
-      r.a = ldg_stream(p + i0);
+      r.v[0] = ldg_stream(p + i0);
     } else {
       uint32_t w[4];
 #pragma unroll
@@ -128,26 +147,26 @@ __device__ __forceinline__ Raw<DT> fetch(const void* row, int i0, int vend, bool
         const uint32_t hi = (e1 < vend) ? (uint32_t)__ldg(p + e1) : 0x7FC0u;
         w[j] = lo | (hi << 16);
       }
-      r.a = make_uint4(w[0], w[1], w[2], w[3]);
+      r.v[0] = make_uint4(w[0], w[1], w[2], w[3]);
     }
   } else {
     const uint32_t* p = (const uint32_t*)row;
     if (aligned && i0 + kPerThread <= vend) {
-      r.a = ldg_stream(p + i0);
-      r.b = ldg_stream(p + i0 + 4);
+      r.v[0] = ldg_stream(p + i0);
+      r.v[1] = ldg_stream(p + i0 + 4);
     } else {
       uint32_t w[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j) w[j] = (i0 + j < vend) ? __ldg(p + i0 + j) : 0x7FC00000u;
-      r.a = make_uint4(w[0], w[1], w[2], w[3]);
-      r.b = make_uint4(w[4], w[5], w[6], w[7]);
+      r.v[0] = make_uint4(w[0], w[1], w[2], w[3]);
+      r.v[1] = make_uint4(w[4], w[5], w[6], w[7]);
     }
   }
   return r;
 }
 
 __device__ __forceinline__ void decode(const Raw<ERSD_BF16>& r, float z[8]) {
-  const uint32_t w[4] = {r.a.x, r.a.y, r.a.z, r.a.w};
+  const uint32_t w[4] = {r.v[0].x, r.v[0].y, r.v[0].z, r.v[0].w};
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
     z[2 * j] = __uint_as_float(w[j] << 16);
@@ -155,10 +174,17 @@ __device__ __forceinline__ void decode(const Raw<ERSD_BF16>& r, float z[8]) {
   }
 }
 __device__ __forceinline__ void decode(const Raw<ERSD_F32>& r, float z[8]) {
-  z[0] = __uint_as_float(r.a.x); z[1] = __uint_as_float(r.a.y);
-  z[2] = __uint_as_float(r.a.z); z[3] = __uint_as_float(r.a.w);
-  z[4] = __uint_as_float(r.b.x); z[5] = __uint_as_float(r.b.y);
-  z[6] = __uint_as_float(r.b.z); z[7] = __uint_as_float(r.b.w);
+  z[0] = __uint_as_float(r.v[0].x); z[1] = __uint_as_float(r.v[0].y);
+  z[2] = __uint_as_float(r.v[0].z); z[3] = __uint_as_float(r.v[0].w);
+  z[4] = __uint_as_float(r.v[1].x); z[5] = __uint_as_float(r.v[1].y);
+  z[6] = __uint_as_float(r.v[1].z); z[7] = __uint_as_float(r.v[1].w);
+}
+
+// Logit j (0..7) of a thread's slice as staged in shared memory.
+template <int DT>
+__device__ __forceinline__ float staged_logit(const uint4* raw, int j) {
+  if constexpr (DT == ERSD_BF16) return __uint_as_float((uint32_t)((const uint16_t*)raw)[j] << 16);
+  else return ((const float*)raw)[j];
 }
 
 // Sorted list of the smallest (key, idx) pairs seen by a warp: lane l holds the l-th smallest.
@@ -183,13 +209,18 @@ struct WarpList {
       idx = i;
     }
   }
-  __device__ __forceinline__ double key_at(int l) const { return __shfl_sync(kFull, key, l); }
 };
 
 // Upper bound, in the screening keys' log2 units, of a double key in natural-log units.
 __device__ __forceinline__ float tau_of_exact(double key) {
   const float t = (float)(key * 1.4426950408889634);
   return fmaf(fabsf(t), 2.384185791015625e-7f, t);
+}
+
+// Value a thread-tile's lower bound (which carries an offset of 32, see stream_tiles) is compared
+// with: everything above it is out of the race for threshold tau.
+__device__ __forceinline__ float lim_of_tau(float tau) {
+  return fmaf(fabsf(tau), 9.5367431640625e-7f, tau) + 32.001953125f;
 }
 
 // c-th smallest of the lanes' values (c >= 1), +inf if fewer than c lanes hold a number.
@@ -205,15 +236,6 @@ __device__ __forceinline__ float cth_smallest(float m, int c, int lane) {
   return (v == 0x7FFFFFFF) ? INFINITY : float_of(v);
 }
 
-// State of one role (target row or draft row) of the block's work item.
-struct Role {
-  const void* row;
-  bool aligned;
-  int c;        // arrivals wanted
-  float tau;    // log2 units: no index whose true key exceeds tau can be among the first c
-  WarpList list;
-};
-
 // Shared-memory float minimum (rare path).
 __device__ __forceinline__ void smem_min(float* addr, float v) {
   float old = *(volatile float*)addr;
@@ -224,11 +246,11 @@ __device__ __forceinline__ void smem_min(float* addr, float v) {
   }
 }
 
-// Upper bound of the eight logits of a tile slice (NaN ignored; NaN if all are NaN).
+// Upper bound of the eight logits of a thread's slice (NaN ignored; NaN if all are NaN).
 __device__ __forceinline__ float logits_upper_bound(const Raw<ERSD_BF16>& r) {
   uint32_t m01, m23, m;
-  asm("max.bf16x2 %0, %1, %2;" : "=r"(m01) : "r"(r.a.x), "r"(r.a.y));
-  asm("max.bf16x2 %0, %1, %2;" : "=r"(m23) : "r"(r.a.z), "r"(r.a.w));
+  asm("max.bf16x2 %0, %1, %2;" : "=r"(m01) : "r"(r.v[0].x), "r"(r.v[0].y));
+  asm("max.bf16x2 %0, %1, %2;" : "=r"(m23) : "r"(r.v[0].z), "r"(r.v[0].w));
   asm("max.bf16x2 %0, %1, %2;" : "=r"(m) : "r"(m01), "r"(m23));
   // The odd elements' maximum sits in the high half.  Read with the low half attached it is
   // off by less than one bf16 ulp (2^-7 relative, towards larger magnitude); widen it to a
@@ -239,115 +261,259 @@ __device__ __forceinline__ float logits_upper_bound(const Raw<ERSD_BF16>& r) {
   return fmaxf(hi_ub, lo);
 }
 __device__ __forceinline__ float logits_upper_bound(const Raw<ERSD_F32>& r) {
-  const float a = fmaxf(fmaxf(__uint_as_float(r.a.x), __uint_as_float(r.a.y)),
-                        fmaxf(__uint_as_float(r.a.z), __uint_as_float(r.a.w)));
-  const float b = fmaxf(fmaxf(__uint_as_float(r.b.x), __uint_as_float(r.b.y)),
-                        fmaxf(__uint_as_float(r.b.z), __uint_as_float(r.b.w)));
+  const float a = fmaxf(fmaxf(__uint_as_float(r.v[0].x), __uint_as_float(r.v[0].y)),
+                        fmaxf(__uint_as_float(r.v[0].z), __uint_as_float(r.v[0].w)));
+  const float b = fmaxf(fmaxf(__uint_as_float(r.v[1].x), __uint_as_float(r.v[1].y)),
+                        fmaxf(__uint_as_float(r.v[1].z), __uint_as_float(r.v[1].w)));
   return fmaxf(a, b);
 }
 
-// Examine eight indices of one role: a[j] = lg[j] - z[j] * c2 is either the screening key
-// (`accurate`: within the slack of the true key, so the c-th smallest lane minimum also
-// tightens tau) or only a lower bound of it.  Indices that can still be among the first c
-// arrivals are evaluated in double precision and inserted into the warp's list.
-__device__ __forceinline__ void race_role(Role& R, const float z[8], const float lg[8],
-                                          const uint32_t xs[8], int i0, float c2, float T,
-                                          float* sm_tau, int lane, bool accurate) {
-  float a[8];
-  float m = INFINITY;
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    a[j] = fmaf(-z[j], c2, lg[j]);
-    m = fminf(m, a[j]);
+// ---------------------------------------------------------------------------------------------
+// block state
+// ---------------------------------------------------------------------------------------------
+struct RoleInfo {
+  const char* row;  // first element of the role's logit row
+  int c;            // arrivals wanted
+  int aligned;      // rows start on 16-byte boundaries
+};
+
+template <int DT>
+struct __align__(16) Shared {
+  // streaming ring: [stage][role][vector][thread], filled by cp.async, each thread reading back
+  // only what it copied itself
+  uint4 ring[Geo<DT>::kStages][2][Geo<DT>::kVec][kThreads];
+  // per warp and role: the smallest (key, id) pairs seen so far, ascending
+  Entry list[2][kWarps][ERSD_MAX_TOP_C];
+  // per warp: a thread's eight Philox words and its logits, handed to the whole warp
+  uint4 stage[kWarps][2 + 2 * Geo<DT>::kVec];
+  PhiloxRow philox;
+  RoleInfo role[2];
+  float tau[2];  // log2 units: no index whose true key exceeds tau[r] can be among the first c
+  alignas(8) float lim[2];  // lim_of_tau(tau[r])
+  int last;
+  int ttok[ERSD_MAX_ROWS], dtok[ERSD_MAX_ROWS];
+  float tkey[ERSD_MAX_ROWS], dkey[ERSD_MAX_ROWS];
+};
+
+// After an insertion into warp `warp`'s list of role r: its c-th key bounds the role's threshold.
+template <int DT>
+__device__ __forceinline__ void publish_threshold(Shared<DT>& sh, int r, int warp, int lane) {
+  const double kc = sh.list[r][warp][sh.role[r].c - 1].key;
+  if (lane == 0 && kc < (double)INFINITY && kc > -(double)INFINITY) {
+    const float tau = tau_of_exact(kc);
+    smem_min(&sh.tau[r], tau);
+    smem_min(&sh.lim[r], lim_of_tau(tau));
   }
-  const float tau_in = fminf(R.tau, *(volatile float*)sm_tau);
-  float tau = tau_in;
-  const bool hit = m <= tau + screen_slack(tau);
-  if (__any_sync(kFull, hit)) {
-    if (accurate) {
-      const float theta = cth_smallest(m, R.c, lane);
-      tau = fminf(tau, theta + screen_slack(theta));
-    }
-    const float lim = tau + screen_slack(tau);
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const bool cand = a[j] <= lim;
-      if (__any_sync(kFull, cand)) {
-        double dk = (double)INFINITY;
-        if (cand) dk = exact_key(xs[j], z[j], T);
-        unsigned act = __ballot_sync(kFull, cand && dk < (double)INFINITY);
-        while (act) {
-          const int src = __ffs(act) - 1;
-          act &= act - 1;
-          const double k = __shfl_sync(kFull, dk, src);
-          const int i = __shfl_sync(kFull, i0, src) + j;
-          R.list.insert(k, i, lane);
-        }
-      }
-    }
-    const double kc = R.list.key_at(R.c - 1);
-    if (kc < (double)INFINITY) tau = fminf(tau, tau_of_exact(kc));
-    if (lane == 0 && tau < tau_in) smem_min(sm_tau, tau);
-  }
-  R.tau = tau;
 }
 
-// Stream one chunk [v0, v1) of a row (NR = 1) or of a draft/target pair (NR = 2).
-//
-// Fast path per thread and tile of eight indices: two Philox calls, the smallest of the eight
-// words, the largest of the eight logits per role, and one comparison per role of
-//     lg2(x_min) - z_max * c2      (a lower bound of all eight keys, shifted by 32)
-// against the block's threshold.  Only when some lane of the warp cannot rule its eight
-// indices out does the warp look at them one by one (race_role).
+// The rare path of a tile.  Lanes whose `bits` are non-zero hold eight indices (starting at i0)
+// that the cheap bound could not rule out for the roles named by the bits.  One such lane at a
+// time hands its words and logits to the warp through shared memory; lanes 0-7 (role 0) and 8-15
+// (role 1) each take one index, form the accurate single-precision key and, if it is within the
+// slack of the threshold, the double-precision key that decides; survivors enter the warp's list.
 template <int DT, int NR>
-__device__ __forceinline__ void stream_chunk(Role* roles, int v0, int v1, const PhiloxRow& pr,
-                                             float c2, float T, bool greedy, float* sm_tau,
-                                             int lane) {
-  const int tid = threadIdx.x;
-  const int ntiles = (v1 - v0 + kTile - 1) / kTile;
-  Raw<DT> cur[NR], nxt[NR];
-  int i0 = v0 + tid * kPerThread;
+__device__ __noinline__ void settle_tile(Shared<DT>* shp, uint4 xa, uint4 xb, Raw<DT> r0, Raw<DT> r1,
+                                         int i0, unsigned bits, float c2, float T) {
+  Shared<DT>& sh = *shp;
+  constexpr int kVec = Geo<DT>::kVec;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const bool greedy = (T == 0.0f);
+  uint4* st = sh.stage[warp];
+  unsigned who = __ballot_sync(kFull, bits != 0);
+  while (who) {
+    const int src = __ffs(who) - 1;
+    who &= who - 1;
+    if (lane == src) {
+      st[0] = xa;
+      st[1] = xb;
 #pragma unroll
-  for (int r = 0; r < NR; ++r) cur[r] = fetch<DT>(roles[r].row, i0, v1, roles[r].aligned);
-  for (int t = 0; t < ntiles; ++t) {
-    const int in = i0 + kTile;
-    if (t + 1 < ntiles) {
-#pragma unroll
-      for (int r = 0; r < NR; ++r) nxt[r] = fetch<DT>(roles[r].row, in, v1, roles[r].aligned);
-    }
-    uint32_t xs[8];
-    pr.words((uint32_t)i0 >> 2, xs);
-    pr.words(((uint32_t)i0 >> 2) + 1u, xs + 4);
-    const uint32_t xm = min(min(min(xs[0], xs[1]), min(xs[2], xs[3])),
-                            min(min(xs[4], xs[5]), min(xs[6], xs[7])));
-    // lg2(w) >= lg2(x) - 32; the 32 moves to the threshold's side.  Greedy rows have no race.
-    const float lgm = greedy ? 32.0f : lg2_fast((float)xm);
-    bool pass = false, boot = false;
-#pragma unroll
-    for (int r = 0; r < NR; ++r) {
-      const float tau = *(volatile float*)(sm_tau + r);
-      const float lim32 = fmaf(fabsf(tau), 9.5367431640625e-7f, tau) + 32.001953125f;
-      const float lb = fmaf(-logits_upper_bound(cur[r]), c2, lgm);
-      pass |= !(lb > lim32);
-      boot |= !(tau < INFINITY);
-    }
-    if (__any_sync(kFull, pass)) {
-      // No threshold yet (first tiles of a chunk): use the accurate screening value so that
-      // the tile itself yields one.  Otherwise the cheaper lower bound lg2(x) - 32 will do.
-      float lg[8];
-#pragma unroll
-      for (int j = 0; j < 8; ++j)
-        lg[j] = greedy ? 0.0f : (boot ? screen_lg2_e(xs[j]) : lg2_fast((float)xs[j]) - 32.0f);
-#pragma unroll
-      for (int r = 0; r < NR; ++r) {
-        float z[8];
-        decode(cur[r], z);
-        race_role(roles[r], z, lg, xs, i0, c2, T, sm_tau + r, lane, boot || greedy);
+      for (int v = 0; v < kVec; ++v) {
+        st[2 + v] = r0.v[v];
+        if (NR == 2) st[2 + kVec + v] = r1.v[v];
       }
     }
+    const int i0s = __shfl_sync(kFull, i0, src);
+    const unsigned bs = __shfl_sync(kFull, bits, src);
+    __syncwarp();
+    const int j = lane & 7, role = lane >> 3;
+    double dk = (double)INFINITY;
+    if (lane < 8 * NR && ((bs >> role) & 1u)) {
+      const uint32_t x = ((const uint32_t*)st)[j];
+      const float z = staged_logit<DT>(st + 2 + role * kVec, j);
+      const float a = fmaf(-z, c2, greedy ? 0.0f : screen_lg2_e(x));
+      const float tau = *(volatile float*)&sh.tau[role];
+      if (a <= tau + screen_slack(tau)) dk = exact_key(x, z, T);
+    }
+    unsigned act = __ballot_sync(kFull, dk < (double)INFINITY);
+    unsigned touched = 0;
+    while (act) {
+      const int s = __ffs(act) - 1;
+      act &= act - 1;
+      const double k = __shfl_sync(kFull, dk, s);
+      const int r = s >> 3;
+      Entry* L = sh.list[r][warp];
+      WarpList w;
+      w.key = L[lane].key;
+      w.idx = L[lane].idx;
+      w.insert(k, i0s + (s & 7), lane);
+      L[lane].key = w.key;
+      L[lane].idx = w.idx;
+      touched |= 1u << r;
+    }
+    __syncwarp();
 #pragma unroll
-    for (int r = 0; r < NR; ++r) cur[r] = nxt[r];
-    i0 = in;
+    for (int r = 0; r < NR; ++r)
+      if ((touched >> r) & 1u) publish_threshold(sh, r, warp, lane);
+  }
+}
+
+// A tile looked at index by index: the first tile of a piece (no threshold exists yet, so the
+// tile must yield one), a ragged last tile, and every tile of rows that are not 16-byte aligned.
+// Per role the c-th smallest of the lanes' best accurate single-precision keys, plus slack, is an
+// upper bound of the c-th smallest true key; everything within the slack of the threshold goes
+// to settle_tile.
+template <int DT, int NR>
+__device__ __noinline__ void edge_tile(Shared<DT>* shp, int i0, int vend, float c2, float T) {
+  Shared<DT>& sh = *shp;
+  const int lane = threadIdx.x & 31;
+  const bool greedy = (T == 0.0f);
+  Raw<DT> raw[2];
+#pragma unroll
+  for (int r = 0; r < NR; ++r) raw[r] = fetch<DT>(sh.role[r].row, i0, vend, sh.role[r].aligned != 0);
+  if (NR == 1) raw[1] = raw[0];
+  uint32_t xs[8];
+  sh.philox.words((uint32_t)i0 >> 2, xs);
+  sh.philox.words(((uint32_t)i0 >> 2) + 1u, xs + 4);
+  float lg[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) lg[j] = greedy ? 0.0f : screen_lg2_e(xs[j]);
+  unsigned bits = 0;
+#pragma unroll
+  for (int r = 0; r < NR; ++r) {
+    float z[8], a[8];
+    decode(raw[r], z);
+    float m = INFINITY;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      a[j] = fmaf(-z[j], c2, lg[j]);
+      m = fminf(m, a[j]);
+    }
+    const float tau_in = *(volatile float*)&sh.tau[r];
+    const float theta = cth_smallest(m, sh.role[r].c, lane);
+    const float tau = fminf(tau_in, theta + screen_slack(theta));
+    if (lane == 0 && tau < tau_in) {
+      smem_min(&sh.tau[r], tau);
+      smem_min(&sh.lim[r], lim_of_tau(tau));
+    }
+    if (m <= tau + screen_slack(tau)) bits |= 1u << r;
+  }
+  __syncwarp();
+  if (__any_sync(kFull, bits != 0))
+    settle_tile<DT, NR>(shp, make_uint4(xs[0], xs[1], xs[2], xs[3]), make_uint4(xs[4], xs[5], xs[6], xs[7]),
+                        raw[0], raw[1], i0, bits, c2, T);
+}
+
+// The streaming loop over `ntiles` full tiles of 16-byte aligned rows; the thread's first index is
+// i0.  Per thread and tile of eight indices: two Philox calls, the smallest of the eight words,
+// the largest of the eight logits per role, and one comparison per role of
+//     lg2(x_min) - z_max * c2      (a lower bound of all eight keys, shifted by 32:
+//                                   lg2(e) >= lg2(w) > lg2(x) - 32)
+// against the block's threshold.  Only when some lane of the warp cannot rule its eight indices
+// out does the warp leave the loop body for settle_tile.  Logits reach the thread through a
+// shared-memory ring that cp.async keeps kStages - 1 tiles ahead.
+template <int DT, int NR>
+struct Streamer {
+  static constexpr int kVec = Geo<DT>::kVec, kStages = Geo<DT>::kStages;
+  static constexpr int kElem = (DT == ERSD_BF16) ? 2 : 4;
+  Shared<DT>* sh;
+  const char* src[NR];  // next tile to request, this thread's slice
+  uint32_t ring0;       // shared-memory address of ring[0][0][0][tid]
+  int requested, ntiles;
+
+  __device__ __forceinline__ void request_one() {
+    if (requested < ntiles) {
+      const uint32_t base = ring0 + (uint32_t)((requested % kStages) * (2 * kVec * kThreads * 16));
+#pragma unroll
+      for (int r = 0; r < NR; ++r) {
+#pragma unroll
+        for (int v = 0; v < kVec; ++v)
+          cp_async16(base + (uint32_t)((r * kVec + v) * kThreads * 16), src[r] + v * 16);
+        src[r] += (size_t)kTile * kElem;
+      }
+    }
+    ++requested;
+    cp_async_commit();
+  }
+
+  // Requests the first kStages - 1 tiles; call before any other work so the copies overlap it.
+  __device__ __forceinline__ void begin(Shared<DT>* shp, int i0, int ntiles_) {
+    sh = shp;
+    ntiles = ntiles_;
+    requested = 0;
+    ring0 = (uint32_t)__cvta_generic_to_shared(&shp->ring[0][0][0][threadIdx.x]);
+#pragma unroll
+    for (int r = 0; r < NR; ++r) src[r] = shp->role[r].row + (size_t)i0 * kElem;
+#pragma unroll
+    for (int s = 0; s < kStages - 1; ++s) request_one();
+  }
+
+  __device__ __forceinline__ void run(int i0, float c2, float T) {
+    const bool greedy = (T == 0.0f);
+    const PhiloxRow pr = sh->philox;
+    uint32_t ctr = (uint32_t)i0 >> 2;
+    const uint32_t lim_addr = (uint32_t)__cvta_generic_to_shared(sh->lim);
+    for (int t = 0; t < ntiles; ++t) {
+      request_one();
+      cp_async_wait<kStages - 1>();
+      Raw<DT> cur[2];
+      const int stage = t % kStages;
+#pragma unroll
+      for (int r = 0; r < NR; ++r)
+#pragma unroll
+        for (int v = 0; v < kVec; ++v) cur[r].v[v] = sh->ring[stage][r][v][threadIdx.x];
+      uint32_t xs[8];
+      pr.words(ctr, xs);
+      pr.words(ctr + 1u, xs + 4);
+      const uint32_t xm = min(__vimin3_u32(xs[0], xs[1], xs[2]),
+                              __vimin3_u32(__vimin3_u32(xs[3], xs[4], xs[5]), xs[6], xs[7]));
+      const float lgm = greedy ? 32.0f : lg2_fast((float)xm);
+      float2 lim;  // both roles' comparison values in one volatile load
+      asm volatile("ld.volatile.shared.v2.f32 {%0,%1}, [%2];" : "=f"(lim.x), "=f"(lim.y) : "r"(lim_addr));
+      unsigned bits = 0;
+      if (!(fmaf(-logits_upper_bound(cur[0]), c2, lgm) > lim.x)) bits |= 1u;
+      if (NR == 2) {
+        if (!(fmaf(-logits_upper_bound(cur[1]), c2, lgm) > lim.y)) bits |= 2u;
+      } else {
+        cur[1] = cur[0];
+      }
+      if (__any_sync(kFull, bits != 0))
+        settle_tile<DT, NR>(sh, make_uint4(xs[0], xs[1], xs[2], xs[3]),
+                            make_uint4(xs[4], xs[5], xs[6], xs[7]), cur[0], cur[1], i0, bits, c2, T);
+      ctr += kTile / 4;
+      i0 += kTile;
+    }
+  }
+};
+
+// One piece = chunk [v0, v1) of a logit row (NR = 1) or of a draft/target pair (NR = 2).
+template <int DT, int NR>
+__device__ __forceinline__ void stream_piece(Shared<DT>* sh, int v0, int v1, float c2, float T) {
+  const int tid = threadIdx.x;
+  bool ring_ok = true;
+#pragma unroll
+  for (int r = 0; r < NR; ++r) ring_ok = ring_ok && (sh->role[r].aligned != 0);
+  const int ntiles = (v1 - v0 + kTile - 1) / kTile;
+  const int nfull = (v1 - v0) / kTile;       // tiles that lie fully inside the piece
+  int i0 = v0 + tid * kPerThread;
+  if (ring_ok) {
+    Streamer<DT, NR> st;
+    st.begin(sh, i0 + kTile, nfull > 1 ? nfull - 1 : 0);
+    edge_tile<DT, NR>(sh, i0, v1, c2, T);     // first tile: yields the first threshold
+    if (nfull > 1) st.run(i0 + kTile, c2, T);
+    cp_async_wait<0>();
+    if (ntiles > 1 && ntiles > nfull) edge_tile<DT, NR>(sh, i0 + (ntiles - 1) * kTile, v1, c2, T);
+  } else {
+    for (int t = 0; t < ntiles; ++t, i0 += kTile) edge_tile<DT, NR>(sh, i0, v1, c2, T);
   }
 }
 
@@ -364,17 +530,13 @@ __device__ __forceinline__ void merge_partials(WarpList& L, const Entry* part, i
 }
 
 #ifndef ERSD_MIN_BLOCKS
-#define ERSD_MIN_BLOCKS 2  // resident blocks per SM the register allocation aims for
+#define ERSD_MIN_BLOCKS 4  // resident blocks per SM the register allocation aims for
 #endif
 
 template <int DT>
 __global__ void __launch_bounds__(kThreads, ERSD_MIN_BLOCKS)
 ersd_race_kernel(const Params p, const __grid_constant__ TreeDesc tree) {
-  __shared__ float sm_tau[2];
-  __shared__ Entry sm_list[2][kWarps][ERSD_MAX_TOP_C];
-  __shared__ int sm_last;
-  __shared__ int sm_ttok[ERSD_MAX_ROWS], sm_dtok[ERSD_MAX_ROWS];
-  __shared__ float sm_tkey[ERSD_MAX_ROWS], sm_dkey[ERSD_MAX_ROWS];
+  __shared__ Shared<DT> sh;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // work item -> (row, sequence, chunk); rows are launched in tree.order so that the heavier
@@ -392,62 +554,57 @@ ersd_race_kernel(const Params p, const __grid_constant__ TreeDesc tree) {
   const int v0 = s * p.per_chunk;
   const int v1 = min(p.V, v0 + p.per_chunk);
 
-  const uint64_t seed = p.seeds[b];
-  const uint32_t seq = p.seq_ids ? p.seq_ids[b] : (uint32_t)b;
-  const uint32_t pos = (p.pos_offsets ? p.pos_offsets[b] : 0u) + (uint32_t)r;
   const float T = p.temps ? p.temps[(int64_t)b * p.ts_b + (int64_t)r * p.ts_r] : p.T;
-  const bool greedy = (T == 0.0f);
-  float c2;
-  if (greedy) c2 = 1.0f;
-  else if (T > 0.0f && T < INFINITY) c2 = (float)(1.4426950408889634 / (double)T);
-  else c2 = __int_as_float(0x7FC00000);  // invalid temperature: no token arrives
-
-  if (tid < 2) sm_tau[tid] = INFINITY;
-  __syncthreads();
-  PhiloxRow pr;
-  pr.init(seed, seq, pos);
+  const bool valid_T = (T >= 0.0f && T < INFINITY);
+  // keys are screened in log2 units: lg2(e) - z * c2 (greedy rows: -z * log2(e), no race)
+  const float c2 = (T == 0.0f) ? kLog2e : (float)(1.4426950408889634 / (double)T);
 
   const size_t es = (DT == ERSD_BF16) ? 2 : 4;
-  Role roles[2];
-  roles[0].row = (const char*)p.target + (size_t)unit * (size_t)p.ld_t * es;
-  roles[0].aligned = p.aligned_t;
-  roles[0].c = c0;
-  roles[0].tau = INFINITY;
-  roles[0].list.init();
-  roles[1].row = nullptr;
-  roles[1].aligned = p.aligned_d;
-  roles[1].c = cq > 0 ? cq : 1;
-  roles[1].tau = INFINITY;
-  roles[1].list.init();
-  if (cq > 0) {
-    roles[1].row = (const char*)p.draft + ((size_t)b * p.draft_rows + r) * (size_t)p.ld_d * es;
-    stream_chunk<DT, 2>(roles, v0, v1, pr, c2, T, greedy, sm_tau, lane);
-  } else {
-    stream_chunk<DT, 1>(roles, v0, v1, pr, c2, T, greedy, sm_tau, lane);
+  if (tid == 0) {
+    const uint64_t seed = p.seeds[b];
+    const uint32_t seq = p.seq_ids ? p.seq_ids[b] : (uint32_t)b;
+    const uint32_t pos = (p.pos_offsets ? p.pos_offsets[b] : 0u) + (uint32_t)r;
+    sh.philox.init(seed, seq, pos);
+    sh.role[0].row = (const char*)p.target + (size_t)unit * (size_t)p.ld_t * es;
+    sh.role[0].c = c0;
+    sh.role[0].aligned = p.aligned_t;
+    sh.role[1].row = cq > 0 ? (const char*)p.draft + ((size_t)b * p.draft_rows + r) * (size_t)p.ld_d * es
+                            : nullptr;
+    sh.role[1].c = cq > 0 ? cq : 1;
+    sh.role[1].aligned = p.aligned_d;
+    sh.tau[0] = sh.tau[1] = INFINITY;
+    sh.lim[0] = sh.lim[1] = INFINITY;
   }
-
-  // ---- block merge: every warp publishes its list, warp `role` merges that role's lists ----
-  const int nroles = cq > 0 ? 2 : 1;
-#pragma unroll
-  for (int role = 0; role < 2; ++role) {
-    if (role >= nroles) break;
+  {
     Entry e;
-    e.key = roles[role].list.key;
-    e.idx = roles[role].list.idx;
+    e.key = (double)INFINITY;
+    e.idx = 0x7FFFFFFF;
     e.pad = 0;
-    sm_list[role][warp][lane] = e;
+    sh.list[0][warp][lane] = e;
+    sh.list[1][warp][lane] = e;
   }
   __syncthreads();
+
+  if (valid_T) {  // a row with an invalid temperature has no arrivals
+    if (cq > 0) stream_piece<DT, 2>(&sh, v0, v1, c2, T);
+    else stream_piece<DT, 1>(&sh, v0, v1, c2, T);
+  }
+  __syncthreads();
+
+  // ---- block merge: warp `role` merges the eight warps' lists of that role ----
+  const int nroles = cq > 0 ? 2 : 1;
   const bool direct = (p.mode == kSample && p.S == 1);
   if (warp < nroles) {
     const int role = warp;
-    const int c = role ? roles[1].c : roles[0].c;
-    WarpList L = role ? roles[1].list : roles[0].list;
-    for (int w = 0; w < kWarps; ++w) {
-      if (w == warp) continue;
+    const int c = sh.role[role].c;
+    WarpList L;
+    L.key = sh.list[role][0][lane].key;
+    L.idx = sh.list[role][0][lane].idx;
+    for (int w = 1; w < kWarps; ++w) {
       for (int e = 0; e < c; ++e) {
-        const Entry en = sm_list[role][w][e];
-        if (en.idx != 0x7FFFFFFF) L.insert(en.key, en.idx, lane);
+        const Entry en = sh.list[role][w][e];
+        if (en.idx == 0x7FFFFFFF) break;
+        L.insert(en.key, en.idx, lane);
       }
     }
     if (direct) {
@@ -474,10 +631,10 @@ ersd_race_kernel(const Params p, const __grid_constant__ TreeDesc tree) {
   const int group_items = (p.mode == kSample) ? p.S : p.rows * p.S;
   if (tid == 0) {
     const int old = atomicAdd(counter, 1);
-    sm_last = (old == group_items - 1);
+    sh.last = (old == group_items - 1);
   }
   __syncthreads();
-  if (!sm_last) return;
+  if (!sh.last) return;
   __threadfence();
   if (tid == 0) *counter = 0;  // leave the workspace ready for the next call
 
@@ -505,19 +662,19 @@ ersd_race_kernel(const Params p, const __grid_constant__ TreeDesc tree) {
     const bool ok = L.idx != 0x7FFFFFFF;
     if (role == 0) {
       if (lane == 0) {
-        sm_ttok[n] = ok ? L.idx : -1;
-        sm_tkey[n] = ok ? (float)L.key : INFINITY;
+        sh.ttok[n] = ok ? L.idx : -1;
+        sh.tkey[n] = ok ? (float)L.key : INFINITY;
       }
     } else if (lane < c) {
       int m = tree.first_child[n];  // the child of rank `lane`
       for (int q = 0; q < lane; ++q) m = tree.next_sib[m];
-      sm_dtok[m] = ok ? L.idx : -1;
-      sm_dkey[m] = ok ? (float)L.key : INFINITY;
+      sh.dtok[m] = ok ? L.idx : -1;
+      sh.dkey[m] = ok ? (float)L.key : INFINITY;
     }
   }
   if (tid == 0) {
-    sm_dtok[0] = -1;
-    sm_dkey[0] = INFINITY;
+    sh.dtok[0] = -1;
+    sh.dkey[0] = INFINITY;
   }
   __syncthreads();
 
@@ -528,17 +685,17 @@ ersd_race_kernel(const Params p, const __grid_constant__ TreeDesc tree) {
   }
   for (int n = tid; n < p.rows; n += kThreads) {
     const size_t o = (size_t)b * p.rows + n;
-    if (p.out_target_tok) p.out_target_tok[o] = sm_ttok[n];
-    if (p.out_target_key) p.out_target_key[o] = sm_tkey[n];
+    if (p.out_target_tok) p.out_target_tok[o] = sh.ttok[n];
+    if (p.out_target_key) p.out_target_key[o] = sh.tkey[n];
     if (p.chain_outputs) {
       if (n >= 1) {
         const size_t od = (size_t)b * (p.rows - 1) + (n - 1);
-        if (p.out_draft_tok) p.out_draft_tok[od] = sm_dtok[n];
-        if (p.out_draft_key) p.out_draft_key[od] = sm_dkey[n];
+        if (p.out_draft_tok) p.out_draft_tok[od] = sh.dtok[n];
+        if (p.out_draft_key) p.out_draft_key[od] = sh.dkey[n];
       }
     } else {
-      if (p.out_draft_tok) p.out_draft_tok[o] = sm_dtok[n];
-      if (p.out_draft_key) p.out_draft_key[o] = sm_dkey[n];
+      if (p.out_draft_tok) p.out_draft_tok[o] = sh.dtok[n];
+      if (p.out_draft_key) p.out_draft_key[o] = sh.dkey[n];
     }
   }
   __syncthreads();
@@ -547,13 +704,13 @@ ersd_race_kernel(const Params p, const __grid_constant__ TreeDesc tree) {
     // token drafted at one of its children.
     int cur = 0, depth = 0;
     for (;;) {
-      const int w = sm_ttok[cur];
+      const int w = sh.ttok[cur];
       p.out_tokens[(size_t)b * cols + depth] = w;
       if (p.out_path) p.out_path[(size_t)b * cols + depth] = cur;
       int next = -1;
       if (w >= 0) {
         for (int m = tree.first_child[cur]; m >= 0; m = tree.next_sib[m]) {
-          if (sm_dtok[m] == w) {
+          if (sh.dtok[m] == w) {
             next = m;
             break;
           }
@@ -579,7 +736,7 @@ __global__ void ersd_row_keys_kernel(const void* row, int V, float T, uint64_t s
   if (mode == 0) {
     out[i] = (float)exact_key(x, z, T);
   } else {
-    const float c2 = (T == 0.0f) ? 1.0f : (float)(1.4426950408889634 / (double)T);
+    const float c2 = (float)(1.4426950408889634 / (T == 0.0f ? 1.0 : (double)T));
     const float lg = (T == 0.0f) ? 0.0f : screen_lg2_e(x);
     out[i] = fmaf(-z, c2, lg) * kLn2;
   }
@@ -724,9 +881,33 @@ static int build_tree(const int32_t* parent, int N, TreeDesc* t, int* depth_out,
   return ERSD_OK;
 }
 
+// Four resident blocks per SM need about 180 KB of shared memory: ask for the largest carveout
+// (a hint to the driver; set once per device and kernel).
+static int prefer_shared_memory() {
+  static std::mutex m;
+  static bool done[64];
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (dev < 0 || dev >= 64) return ERSD_EUNSUPPORTED;
+  std::lock_guard<std::mutex> lock(m);
+  if (!done[dev]) {
+    e = cudaFuncSetAttribute(ersd_race_kernel<ERSD_BF16>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                             cudaSharedmemCarveoutMaxShared);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(ersd_race_kernel<ERSD_F32>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                               cudaSharedmemCarveoutMaxShared);
+    if (e != cudaSuccess) return cuda_fail(e);
+    done[dev] = true;
+  }
+  return ERSD_OK;
+}
+
 static int launch(const Params& p, const TreeDesc& tree, int dt, cudaStream_t st) {
   const int64_t items = (int64_t)p.B * p.rows * p.S;
   if (items > 0x7FFFFFFF) return ERSD_EINVAL;
+  const int pst = prefer_shared_memory();
+  if (pst != ERSD_OK) return pst;
   if (dt == ERSD_BF16) ersd_race_kernel<ERSD_BF16><<<(unsigned)items, kThreads, 0, st>>>(p, tree);
   else ersd_race_kernel<ERSD_F32><<<(unsigned)items, kThreads, 0, st>>>(p, tree);
   const cudaError_t e = cudaGetLastError();
