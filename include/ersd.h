@@ -204,7 +204,10 @@ int ersd_tree_depth(const int32_t* parent, int N);
  * natural-log units): out_keys[i], i < V, device float32.
  *   mode 0: the double-precision evaluation the library uses to decide winners;
  *   mode 1: the single-precision screening value it uses to discard losers
- *           (within about 1e-3 of mode 0 for |key| up to a few hundred).
+ *           (within about 1e-3 of mode 0 for |key| up to a few hundred);
+ *   mode 2: (mode-0 key minus the same key formed with the CUDA math library's
+ *           log and log1p) * 1e12 -- checks the library's own straight-line
+ *           double-precision logarithm on the device.
  */
 int ersd_row_keys(const void* row_logits, ersd_dtype dt, int V, float T, uint64_t seed,
                   uint32_t seq_id, uint32_t position, int mode, float* out_keys, void* cuda_stream);

@@ -19,6 +19,10 @@
 #include "ersd.h"
 #include "ersd_math.cuh"
 
+#ifndef ERSD_MIN_BLOCKS
+#define ERSD_MIN_BLOCKS 4  // resident blocks per SM the register allocation aims for
+#endif
+
 namespace ersd {
 
 constexpr int kThreads = 256;
@@ -41,7 +45,8 @@ struct Entry {  // one arrival: race key (natural-log units) and token id
 // zero when a call starts; partial lists are always rewritten before they are read).
 struct Slot {
   int counter;  // arrivals of the group whose first row this is; reset to 0 by the last arrival
-  int pad[3];
+  unsigned tau_code[2];  // per role: best threshold published so far (0 = none), see code_of_tau
+  int pad;
   Entry part[2][kPartCap];  // per role: S partial lists of c entries each
 };
 
@@ -223,6 +228,13 @@ __device__ __forceinline__ float lim_of_tau(float tau) {
   return fmaf(fabsf(tau), 9.5367431640625e-7f, tau) + 32.001953125f;
 }
 
+// Thresholds travel between the chunks of a row through the workspace as unsigned codes that
+// grow as the threshold falls, with 0 (the workspace's resting state) meaning "none yet".
+__device__ __forceinline__ unsigned code_of_tau(float tau) { return (unsigned)ord_of(-tau) ^ 0x80000000u; }
+__device__ __forceinline__ float tau_of_code(unsigned code) {
+  return code == 0u ? INFINITY : -float_of((int)(code ^ 0x80000000u));
+}
+
 // c-th smallest of the lanes' values (c >= 1), +inf if fewer than c lanes hold a number.
 __device__ __forceinline__ float cth_smallest(float m, int c, int lane) {
   int o = (m == m) ? ord_of(m) : 0x7FFFFFFF;
@@ -284,9 +296,8 @@ struct __align__(16) Shared {
   uint4 ring[Geo<DT>::kStages][2][Geo<DT>::kVec][kThreads];
   // per warp and role: the smallest (key, id) pairs seen so far, ascending
   Entry list[2][kWarps][ERSD_MAX_TOP_C];
-  // per warp: a thread's eight Philox words and its logits, handed to the whole warp
-  uint4 stage[kWarps][2 + 2 * Geo<DT>::kVec];
   PhiloxRow philox;
+  double inv_T;  // 1 / T of the row being raced (0 for greedy rows)
   RoleInfo role[2];
   float tau[2];  // log2 units: no index whose true key exceeds tau[r] can be among the first c
   alignas(8) float lim[2];  // lim_of_tau(tau[r])
@@ -306,43 +317,45 @@ __device__ __forceinline__ void publish_threshold(Shared<DT>& sh, int r, int war
   }
 }
 
-// The rare path of a tile.  Lanes whose `bits` are non-zero hold eight indices (starting at i0)
-// that the cheap bound could not rule out for the roles named by the bits.  One such lane at a
-// time hands its words and logits to the warp through shared memory; lanes 0-7 (role 0) and 8-15
-// (role 1) each take one index, form the accurate single-precision key and, if it is within the
-// slack of the threshold, the double-precision key that decides; survivors enter the warp's list.
-template <int DT, int NR>
-__device__ __noinline__ void settle_tile(Shared<DT>* shp, uint4 xa, uint4 xb, Raw<DT> r0, Raw<DT> r1,
-                                         int i0, unsigned bits, float c2, float T) {
+// Logit j (0..7) of thread `t`'s slice of role `role` in ring stage `stage`.
+template <int DT>
+__device__ __forceinline__ float ring_logit(const Shared<DT>& sh, int stage, int role, int t, int j) {
+  if constexpr (DT == ERSD_BF16) {
+    return __uint_as_float((uint32_t)((const uint16_t*)&sh.ring[stage][role][0][t])[j] << 16);
+  } else {
+    return ((const float*)&sh.ring[stage][role][j >> 2][t])[j & 3];
+  }
+}
+
+// The rare path of a tile.  Lanes whose `bits` are non-zero own eight indices (starting at their
+// i0, logits in ring stage `stage`) that the cheap bound could not rule out for the roles named
+// by the bits.  One such lane at a time is served by the warp: lanes 0-7 (role 0) and 8-15
+// (role 1) each take one index, draw its Philox word again, form the accurate single-precision
+// key and, if it is within the slack of the threshold, the double-precision key that decides;
+// survivors enter the warp's list.
+template <int DT>
+__device__ __noinline__ void settle_tile(Shared<DT>* shp, int stage, int i0, unsigned bits, float c2,
+                                         float T) {
   Shared<DT>& sh = *shp;
-  constexpr int kVec = Geo<DT>::kVec;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const bool greedy = (T == 0.0f);
-  uint4* st = sh.stage[warp];
+  __syncwarp();  // every lane's ring slot is complete and visible to the warp
   unsigned who = __ballot_sync(kFull, bits != 0);
   while (who) {
     const int src = __ffs(who) - 1;
     who &= who - 1;
-    if (lane == src) {
-      st[0] = xa;
-      st[1] = xb;
-#pragma unroll
-      for (int v = 0; v < kVec; ++v) {
-        st[2 + v] = r0.v[v];
-        if (NR == 2) st[2 + kVec + v] = r1.v[v];
-      }
-    }
     const int i0s = __shfl_sync(kFull, i0, src);
     const unsigned bs = __shfl_sync(kFull, bits, src);
-    __syncwarp();
-    const int j = lane & 7, role = lane >> 3;
+    const int j = lane & 7, role = (lane >> 3) & 1;
     double dk = (double)INFINITY;
-    if (lane < 8 * NR && ((bs >> role) & 1u)) {
-      const uint32_t x = ((const uint32_t*)st)[j];
-      const float z = staged_logit<DT>(st + 2 + role * kVec, j);
+    if (lane < 16 && ((bs >> role) & 1u)) {
+      uint32_t w[4];
+      sh.philox.words(((uint32_t)i0s >> 2) + (uint32_t)(j >> 2), w);
+      const uint32_t x = (j & 2) ? ((j & 1) ? w[3] : w[2]) : ((j & 1) ? w[1] : w[0]);
+      const float z = ring_logit<DT>(sh, stage, role, warp * 32 + src, j);
       const float a = fmaf(-z, c2, greedy ? 0.0f : screen_lg2_e(x));
       const float tau = *(volatile float*)&sh.tau[role];
-      if (a <= tau + screen_slack(tau)) dk = exact_key(x, z, T);
+      if (a <= tau + screen_slack(tau)) dk = exact_key(x, z, sh.inv_T, greedy);
     }
     unsigned act = __ballot_sync(kFull, dk < (double)INFINITY);
     unsigned touched = 0;
@@ -352,35 +365,39 @@ __device__ __noinline__ void settle_tile(Shared<DT>* shp, uint4 xa, uint4 xb, Ra
       const double k = __shfl_sync(kFull, dk, s);
       const int r = s >> 3;
       Entry* L = sh.list[r][warp];
-      WarpList w;
-      w.key = L[lane].key;
-      w.idx = L[lane].idx;
-      w.insert(k, i0s + (s & 7), lane);
-      L[lane].key = w.key;
-      L[lane].idx = w.idx;
+      WarpList wl;
+      wl.key = L[lane].key;
+      wl.idx = L[lane].idx;
+      wl.insert(k, i0s + (s & 7), lane);
+      L[lane].key = wl.key;
+      L[lane].idx = wl.idx;
       touched |= 1u << r;
     }
     __syncwarp();
-#pragma unroll
-    for (int r = 0; r < NR; ++r)
-      if ((touched >> r) & 1u) publish_threshold(sh, r, warp, lane);
+    if (touched & 1u) publish_threshold(sh, 0, warp, lane);
+    if (touched & 2u) publish_threshold(sh, 1, warp, lane);
   }
+  __syncwarp();  // nobody overwrites a ring slot that a lane is still reading
 }
 
-// A tile looked at index by index: the first tile of a piece (no threshold exists yet, so the
-// tile must yield one), a ragged last tile, and every tile of rows that are not 16-byte aligned.
-// Per role the c-th smallest of the lanes' best accurate single-precision keys, plus slack, is an
-// upper bound of the c-th smallest true key; everything within the slack of the threshold goes
-// to settle_tile.
+// A tile looked at index by index: the first tile of a piece when no threshold exists yet (the
+// tile must yield one), a ragged last tile, and every tile of rows that are not 16-byte
+// aligned.  Per role the c-th smallest of the lanes' best accurate single-precision keys, plus
+// slack, is an upper bound of the c-th smallest true key; everything within the slack of the
+// threshold goes to settle_tile, which finds the logits in ring stage `stage` (free at these
+// moments: the streaming loop has no copy in flight into it).
 template <int DT, int NR>
-__device__ __noinline__ void edge_tile(Shared<DT>* shp, int i0, int vend, float c2, float T) {
+__device__ __noinline__ void edge_tile(Shared<DT>* shp, int stage, int i0, int vend, float c2, float T) {
   Shared<DT>& sh = *shp;
   const int lane = threadIdx.x & 31;
   const bool greedy = (T == 0.0f);
-  Raw<DT> raw[2];
+  Raw<DT> raw[NR];
 #pragma unroll
-  for (int r = 0; r < NR; ++r) raw[r] = fetch<DT>(sh.role[r].row, i0, vend, sh.role[r].aligned != 0);
-  if (NR == 1) raw[1] = raw[0];
+  for (int r = 0; r < NR; ++r) {
+    raw[r] = fetch<DT>(sh.role[r].row, i0, vend, sh.role[r].aligned != 0);
+#pragma unroll
+    for (int v = 0; v < Geo<DT>::kVec; ++v) sh.ring[stage][r][v][threadIdx.x] = raw[r].v[v];
+  }
   uint32_t xs[8];
   sh.philox.words((uint32_t)i0 >> 2, xs);
   sh.philox.words(((uint32_t)i0 >> 2) + 1u, xs + 4);
@@ -390,14 +407,11 @@ __device__ __noinline__ void edge_tile(Shared<DT>* shp, int i0, int vend, float 
   unsigned bits = 0;
 #pragma unroll
   for (int r = 0; r < NR; ++r) {
-    float z[8], a[8];
+    float z[8];
     decode(raw[r], z);
     float m = INFINITY;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      a[j] = fmaf(-z[j], c2, lg[j]);
-      m = fminf(m, a[j]);
-    }
+    for (int j = 0; j < 8; ++j) m = fminf(m, fmaf(-z[j], c2, lg[j]));
     const float tau_in = *(volatile float*)&sh.tau[r];
     const float theta = cth_smallest(m, sh.role[r].c, lane);
     const float tau = fminf(tau_in, theta + screen_slack(theta));
@@ -408,9 +422,7 @@ __device__ __noinline__ void edge_tile(Shared<DT>* shp, int i0, int vend, float 
     if (m <= tau + screen_slack(tau)) bits |= 1u << r;
   }
   __syncwarp();
-  if (__any_sync(kFull, bits != 0))
-    settle_tile<DT, NR>(shp, make_uint4(xs[0], xs[1], xs[2], xs[3]), make_uint4(xs[4], xs[5], xs[6], xs[7]),
-                        raw[0], raw[1], i0, bits, c2, T);
+  if (__any_sync(kFull, bits != 0)) settle_tile<DT>(shp, stage, i0, bits, c2, T);
 }
 
 // The streaming loop over `ntiles` full tiles of 16-byte aligned rows; the thread's first index is
@@ -425,14 +437,13 @@ template <int DT, int NR>
 struct Streamer {
   static constexpr int kVec = Geo<DT>::kVec, kStages = Geo<DT>::kStages;
   static constexpr int kElem = (DT == ERSD_BF16) ? 2 : 4;
-  Shared<DT>* sh;
+  static constexpr uint32_t kStageBytes = 2 * kVec * kThreads * 16;
   const char* src[NR];  // next tile to request, this thread's slice
-  uint32_t ring0;       // shared-memory address of ring[0][0][0][tid]
   int requested, ntiles;
 
-  __device__ __forceinline__ void request_one() {
+  __device__ __forceinline__ void request_one(uint32_t ring0) {
     if (requested < ntiles) {
-      const uint32_t base = ring0 + (uint32_t)((requested % kStages) * (2 * kVec * kThreads * 16));
+      const uint32_t base = ring0 + (uint32_t)(requested % kStages) * kStageBytes;
 #pragma unroll
       for (int r = 0; r < NR; ++r) {
 #pragma unroll
@@ -446,74 +457,81 @@ struct Streamer {
   }
 
   // Requests the first kStages - 1 tiles; call before any other work so the copies overlap it.
-  __device__ __forceinline__ void begin(Shared<DT>* shp, int i0, int ntiles_) {
-    sh = shp;
+  __device__ __forceinline__ void begin(Shared<DT>* sh, int i0, int ntiles_) {
     ntiles = ntiles_;
     requested = 0;
-    ring0 = (uint32_t)__cvta_generic_to_shared(&shp->ring[0][0][0][threadIdx.x]);
+    const uint32_t ring0 = (uint32_t)__cvta_generic_to_shared(&sh->ring[0][0][0][threadIdx.x]);
 #pragma unroll
-    for (int r = 0; r < NR; ++r) src[r] = shp->role[r].row + (size_t)i0 * kElem;
+    for (int r = 0; r < NR; ++r) src[r] = sh->role[r].row + (size_t)i0 * kElem;
 #pragma unroll
-    for (int s = 0; s < kStages - 1; ++s) request_one();
+    for (int s = 0; s < kStages - 1; ++s) request_one(ring0);
   }
 
-  __device__ __forceinline__ void run(int i0, float c2, float T) {
+  __device__ __forceinline__ void run(Shared<DT>* sh, int i0, float c2, float T) {
     const bool greedy = (T == 0.0f);
     const PhiloxRow pr = sh->philox;
-    uint32_t ctr = (uint32_t)i0 >> 2;
+    const uint32_t ring0 = (uint32_t)__cvta_generic_to_shared(&sh->ring[0][0][0][threadIdx.x]);
     const uint32_t lim_addr = (uint32_t)__cvta_generic_to_shared(sh->lim);
     for (int t = 0; t < ntiles; ++t) {
-      request_one();
+      request_one(ring0);
       cp_async_wait<kStages - 1>();
-      Raw<DT> cur[2];
       const int stage = t % kStages;
+      float zub[NR];
 #pragma unroll
-      for (int r = 0; r < NR; ++r)
+      for (int r = 0; r < NR; ++r) {
+        Raw<DT> cur;
 #pragma unroll
-        for (int v = 0; v < kVec; ++v) cur[r].v[v] = sh->ring[stage][r][v][threadIdx.x];
+        for (int v = 0; v < kVec; ++v) cur.v[v] = sh->ring[stage][r][v][threadIdx.x];
+        zub[r] = logits_upper_bound(cur);
+      }
       uint32_t xs[8];
-      pr.words(ctr, xs);
-      pr.words(ctr + 1u, xs + 4);
+      pr.words((uint32_t)i0 >> 2, xs);
+      pr.words(((uint32_t)i0 >> 2) + 1u, xs + 4);
       const uint32_t xm = min(__vimin3_u32(xs[0], xs[1], xs[2]),
                               __vimin3_u32(__vimin3_u32(xs[3], xs[4], xs[5]), xs[6], xs[7]));
       const float lgm = greedy ? 32.0f : lg2_fast((float)xm);
       float2 lim;  // both roles' comparison values in one volatile load
       asm volatile("ld.volatile.shared.v2.f32 {%0,%1}, [%2];" : "=f"(lim.x), "=f"(lim.y) : "r"(lim_addr));
       unsigned bits = 0;
-      if (!(fmaf(-logits_upper_bound(cur[0]), c2, lgm) > lim.x)) bits |= 1u;
+      if (!(fmaf(-zub[0], c2, lgm) > lim.x)) bits |= 1u;
       if (NR == 2) {
-        if (!(fmaf(-logits_upper_bound(cur[1]), c2, lgm) > lim.y)) bits |= 2u;
-      } else {
-        cur[1] = cur[0];
+        if (!(fmaf(-zub[NR - 1], c2, lgm) > lim.y)) bits |= 2u;
       }
-      if (__any_sync(kFull, bits != 0))
-        settle_tile<DT, NR>(sh, make_uint4(xs[0], xs[1], xs[2], xs[3]),
-                            make_uint4(xs[4], xs[5], xs[6], xs[7]), cur[0], cur[1], i0, bits, c2, T);
-      ctr += kTile / 4;
+      if (__any_sync(kFull, bits != 0)) settle_tile<DT>(sh, stage, i0, bits, c2, T);
       i0 += kTile;
     }
   }
 };
 
-// One piece = chunk [v0, v1) of a logit row (NR = 1) or of a draft/target pair (NR = 2).
+// One piece = chunk [v0, v1) of a logit row (NR = 1) or of a draft/target pair (NR = 2).  When
+// the piece starts with a threshold for every role (handed down by an earlier piece of the same
+// row) all full tiles go through the streaming loop; otherwise the first tile is looked at index
+// by index to produce one.
 template <int DT, int NR>
-__device__ __forceinline__ void stream_piece(Shared<DT>* sh, int v0, int v1, float c2, float T) {
+__device__ __noinline__ void stream_piece(Shared<DT>* sh, int v0, int v1, float c2, float T) {
+  constexpr int kStages = Geo<DT>::kStages;
   const int tid = threadIdx.x;
-  bool ring_ok = true;
+  bool ring_ok = true, have_tau = true;
 #pragma unroll
-  for (int r = 0; r < NR; ++r) ring_ok = ring_ok && (sh->role[r].aligned != 0);
+  for (int r = 0; r < NR; ++r) {
+    ring_ok = ring_ok && (sh->role[r].aligned != 0);
+    have_tau = have_tau && (sh->tau[r] < INFINITY);
+  }
   const int ntiles = (v1 - v0 + kTile - 1) / kTile;
   const int nfull = (v1 - v0) / kTile;       // tiles that lie fully inside the piece
   int i0 = v0 + tid * kPerThread;
   if (ring_ok) {
+    const int first = have_tau ? 0 : 1;      // first tile of the streaming loop
     Streamer<DT, NR> st;
-    st.begin(sh, i0 + kTile, nfull > 1 ? nfull - 1 : 0);
-    edge_tile<DT, NR>(sh, i0, v1, c2, T);     // first tile: yields the first threshold
-    if (nfull > 1) st.run(i0 + kTile, c2, T);
+    st.begin(sh, i0 + first * kTile, nfull > first ? nfull - first : 0);
+    // no threshold yet: the first tile yields one (the requests above leave the last stage free)
+    if (!have_tau) edge_tile<DT, NR>(sh, kStages - 1, i0, v1, c2, T);
+    if (nfull > first) st.run(sh, i0 + first * kTile, c2, T);
     cp_async_wait<0>();
-    if (ntiles > 1 && ntiles > nfull) edge_tile<DT, NR>(sh, i0 + (ntiles - 1) * kTile, v1, c2, T);
+    if (ntiles > nfull && (have_tau || ntiles > 1))
+      edge_tile<DT, NR>(sh, 0, i0 + (ntiles - 1) * kTile, v1, c2, T);
   } else {
-    for (int t = 0; t < ntiles; ++t, i0 += kTile) edge_tile<DT, NR>(sh, i0, v1, c2, T);
+    for (int t = 0; t < ntiles; ++t, i0 += kTile) edge_tile<DT, NR>(sh, 0, i0, v1, c2, T);
   }
 }
 
@@ -529,23 +547,21 @@ __device__ __forceinline__ void merge_partials(WarpList& L, const Entry* part, i
   }
 }
 
-#ifndef ERSD_MIN_BLOCKS
-#define ERSD_MIN_BLOCKS 4  // resident blocks per SM the register allocation aims for
-#endif
-
 template <int DT>
 __global__ void __launch_bounds__(kThreads, ERSD_MIN_BLOCKS)
 ersd_race_kernel(const Params p, const __grid_constant__ TreeDesc tree) {
   __shared__ Shared<DT> sh;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  // work item -> (row, sequence, chunk); rows are launched in tree.order so that the heavier
-  // paired rows start first
-  const int per_row = p.B * p.S;
-  const int ri = blockIdx.x / per_row;
-  const int rem = blockIdx.x - ri * per_row;
-  const int b = rem / p.S;
-  const int s = rem - b * p.S;
+  // work item -> (chunk, row, sequence), chunk-major: every row's first chunk is scheduled
+  // before any second chunk, so that later chunks of a row usually start with the threshold
+  // an earlier one left in the workspace; within a chunk index rows follow tree.order (the
+  // heavier paired rows first)
+  const int n_units = p.B * p.rows;
+  const int s = blockIdx.x / n_units;
+  const int rem = blockIdx.x - s * n_units;
+  const int ri = rem / p.B;
+  const int b = rem - ri * p.B;
   const int r = (p.mode == kSample) ? ri : (int)tree.order[ri];
   const int unit = b * p.rows + r;
 
@@ -565,6 +581,7 @@ ersd_race_kernel(const Params p, const __grid_constant__ TreeDesc tree) {
     const uint32_t seq = p.seq_ids ? p.seq_ids[b] : (uint32_t)b;
     const uint32_t pos = (p.pos_offsets ? p.pos_offsets[b] : 0u) + (uint32_t)r;
     sh.philox.init(seed, seq, pos);
+    sh.inv_T = (T == 0.0f) ? 0.0 : 1.0 / (double)T;
     sh.role[0].row = (const char*)p.target + (size_t)unit * (size_t)p.ld_t * es;
     sh.role[0].c = c0;
     sh.role[0].aligned = p.aligned_t;
@@ -572,8 +589,13 @@ ersd_race_kernel(const Params p, const __grid_constant__ TreeDesc tree) {
                             : nullptr;
     sh.role[1].c = cq > 0 ? cq : 1;
     sh.role[1].aligned = p.aligned_d;
-    sh.tau[0] = sh.tau[1] = INFINITY;
-    sh.lim[0] = sh.lim[1] = INFINITY;
+    // thresholds handed down by earlier chunks of this row (any of them is a valid bound)
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      const float tau = (p.S > 1) ? tau_of_code(__ldcg(&p.slots[unit].tau_code[q])) : INFINITY;
+      sh.tau[q] = tau;
+      sh.lim[q] = (tau < INFINITY) ? lim_of_tau(tau) : INFINITY;
+    }
   }
   {
     Entry e;
@@ -614,12 +636,17 @@ ersd_race_kernel(const Params p, const __grid_constant__ TreeDesc tree) {
         p.out_tokens[o] = ok ? L.idx : -1;
         if (p.out_key) p.out_key[o] = ok ? (float)L.key : INFINITY;
       }
-    } else if (lane < c) {
-      Entry e;
-      e.key = L.key;
-      e.idx = L.idx;
-      e.pad = 0;
-      p.slots[unit].part[role][s * c + lane] = e;
+    } else {
+      if (lane < c) {
+        Entry e;
+        e.key = L.key;
+        e.idx = L.idx;
+        e.pad = 0;
+        p.slots[unit].part[role][s * c + lane] = e;
+      }
+      // hand the threshold down to the row's later chunks
+      const float tau = sh.tau[role];
+      if (lane == 0 && tau < INFINITY) atomicMax(&p.slots[unit].tau_code[role], code_of_tau(tau));
     }
   }
   if (direct) return;
@@ -636,7 +663,13 @@ ersd_race_kernel(const Params p, const __grid_constant__ TreeDesc tree) {
   __syncthreads();
   if (!sh.last) return;
   __threadfence();
-  if (tid == 0) *counter = 0;  // leave the workspace ready for the next call
+  // leave the workspace ready for the next call
+  if (tid == 0) *counter = 0;
+  if (p.mode == kSample) {
+    if (tid < 2) p.slots[unit].tau_code[tid] = 0u;
+  } else {
+    for (int n = tid; n < p.rows * 2; n += kThreads) p.slots[b * p.rows + (n >> 1)].tau_code[n & 1] = 0u;
+  }
 
   if (p.mode == kSample) {
     if (warp == 0) {
@@ -735,6 +768,11 @@ __global__ void ersd_row_keys_kernel(const void* row, int V, float T, uint64_t s
   const uint32_t x = token_word(seed, seq, pos, (uint32_t)i);
   if (mode == 0) {
     out[i] = (float)exact_key(x, z, T);
+  } else if (mode == 2) {
+    // the deciding key against the CUDA math library's log / log1p, in units of 1e-12
+    const double w = ((double)x + 0.5) * (1.0 / 4294967296.0);
+    const double ref = (T == 0.0f) ? -(double)z : log(-log1p(-w)) - (double)z / (double)T;
+    out[i] = (float)((exact_key(x, z, T) - ref) * 1e12);
   } else {
     const float c2 = (float)(1.4426950408889634 / (T == 0.0f ? 1.0 : (double)T));
     const float lg = (T == 0.0f) ? 0.0f : screen_lg2_e(x);
@@ -818,19 +856,30 @@ static bool rows_aligned(const void* base, int64_t ld, int dt) {
   return ((uintptr_t)base & 15) == 0 && ((ld * elem_size(dt)) & 15) == 0;
 }
 
-// Thread blocks per row: enough work items to fill the GPU, chunks of at least four tiles.
+#ifndef ERSD_WAVES
+#define ERSD_WAVES 3            // work items per resident-block slot that the default split aims for
+#endif
+#ifndef ERSD_MIN_CHUNK_TILES
+#define ERSD_MIN_CHUNK_TILES 8  // smallest chunk of a row that the default split makes
+#endif
+
+// Thread blocks per row.  Many more work items than resident blocks, so that the hardware's
+// block scheduler evens out rows of different cost and the last wave is short; chunks stay long
+// enough to amortise a block's set-up and merge.
 static int choose_split(const ersd_opts& o, int64_t units, int V, int cmax) {
   int smax = kPartCap / cmax;
   if (smax > ERSD_MAX_SPLIT) smax = ERSD_MAX_SPLIT;
-  const int by_v = (V + 4 * kTile - 1) / (4 * kTile);
-  if (smax > by_v) smax = by_v;
   if (smax < 1) smax = 1;
+  const int ntiles = (V + kTile - 1) / kTile;
   int S;
   if (o.split_v) {
     S = (int)o.split_v;
+    if (S > ntiles) S = ntiles;
   } else {
-    const int64_t slots = 148 * 4;
-    S = (int)((slots + units - 1) / units);
+    const int64_t slots = 148 * ERSD_MIN_BLOCKS;
+    S = (int)((ERSD_WAVES * slots + units - 1) / units);
+    const int by_v = ntiles / ERSD_MIN_CHUNK_TILES;
+    if (S > by_v) S = by_v;
   }
   if (S > smax) S = smax;
   if (S < 1) S = 1;
@@ -1118,7 +1167,7 @@ int ersd_tree_depth(const int32_t* parent, int N) {
 
 int ersd_row_keys(const void* row_logits, ersd_dtype dt, int V, float T, uint64_t seed,
                   uint32_t seq_id, uint32_t position, int mode, float* out_keys, void* cuda_stream) {
-  if (!row_logits || !out_keys || V < 1 || !temp_ok(T) || (mode != 0 && mode != 1)) return ERSD_EINVAL;
+  if (!row_logits || !out_keys || V < 1 || !temp_ok(T) || (mode < 0 || mode > 2)) return ERSD_EINVAL;
   if (dt != ERSD_F32 && dt != ERSD_BF16) return ERSD_EINVAL;
   if (((uintptr_t)row_logits & (elem_size(dt) - 1)) != 0 || ((uintptr_t)out_keys & 3) != 0)
     return ERSD_EALIGN;

@@ -4,6 +4,7 @@
 #pragma once
 #include <math.h>
 #include <stdint.h>
+#include <string.h>
 
 #if defined(__CUDACC__)
 #define ERSD_HD __host__ __device__ __forceinline__
@@ -122,18 +123,93 @@ ERSD_HD float lg2_fast(float a) {
 #endif
 }
 
-// ln(e) for e = -log1p(-w), w = (x + 1/2) 2^-32, in double precision.  This is
-// the value that decides winners.
-ERSD_HD double exact_ln_e(uint32_t x) {
-  const double w = ((double)x + 0.5) * (1.0 / 4294967296.0);
-  return log(-log1p(-w));
+// 1 / d for d in [1, 4], to double precision: hardware seed and three Newton steps on the
+// device (each squares the relative error), a plain division on the host.
+ERSD_HD double recip_1_4(double d) {
+#if defined(__CUDA_ARCH__)
+  double r;
+  asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(r) : "d"(d));
+  double e = fma(-d, r, 1.0);
+  r = fma(r, e, r);
+  e = fma(-d, r, 1.0);
+  r = fma(r, e, r);
+  e = fma(-d, r, 1.0);
+  r = fma(r, e, r);
+  return r;
+#else
+  return 1.0 / d;
+#endif
 }
 
-// Exact race key in natural-log units; greedy rows (T == 0) use -z.
-ERSD_HD double exact_key(uint32_t x, float z, float T) {
+ERSD_HD double bits_to_double(uint64_t b) {
+#if defined(__CUDA_ARCH__)
+  return __longlong_as_double((long long)b);
+#else
+  double d;
+  memcpy(&d, &b, sizeof d);
+  return d;
+#endif
+}
+ERSD_HD uint64_t double_to_bits(double d) {
+#if defined(__CUDA_ARCH__)
+  return (uint64_t)__double_as_longlong(d);
+#else
+  uint64_t b;
+  memcpy(&b, &d, sizeof b);
+  return b;
+#endif
+}
+
+// atanh(s) / s - 1 = s^2/3 + s^4/5 + ... truncated after s^(2 N); for |s| <= 1/3 and N = 16
+// (resp. |s| <= 0.1716 and N = 10) the truncation is below 2^-56 of the sum.
+template <int N>
+ERSD_HD double atanh_tail(double s2) {
+  double p = 1.0 / (2 * N + 1);
+#pragma unroll
+  for (int n = N - 1; n >= 1; --n) p = fma(p, s2, 1.0 / (2 * n + 1));
+  return p * s2;
+}
+
+// ln(u) for a positive normal double, straight-line: u = m 2^k with m in [sqrt(1/2), sqrt(2)),
+// ln m = 2 atanh((m - 1) / (m + 1)).  A few ulp; no special cases (callers keep u in range).
+ERSD_HD double ln_pos(double u) {
+  uint64_t b = double_to_bits(u);
+  const int32_t hi = (int32_t)(b >> 32);
+  const int32_t k = (hi - 0x3FE6A09E) >> 20;  // high word of sqrt(1/2); arithmetic shift = floor
+  b -= (uint64_t)((int64_t)k << 52);
+  const double m = bits_to_double(b);
+  const double s = (m - 1.0) * recip_1_4(m + 1.0);
+  const double lnm = 2.0 * fma(s, atanh_tail<10>(s * s), s);
+  return fma((double)k, 0.6931471805599453, lnm);
+}
+
+// ln(e) for e = -log1p(-w), w = (x + 1/2) 2^-32, in double precision (a few 1e-16 relative in
+// e, below 1e-14 absolute in ln e).  This is the value that decides winners.
+//   x <  2^31:  -log1p(-w) = 2 atanh(w / (2 - w)),   w / (2 - w) <= 1/3
+//   x >= 2^31:  1 - w = (~x + 1/2) 2^-32 exactly,    e = -ln(1 - w)
+ERSD_HD double exact_ln_e(uint32_t x) {
+  double e;
+  if ((int32_t)x >= 0) {
+    const double w = ((double)x + 0.5) * (1.0 / 4294967296.0);
+    const double s = w * recip_1_4(2.0 - w);
+    e = 2.0 * fma(s, atanh_tail<16>(s * s), s);
+  } else {
+    const double v = ((double)(~x) + 0.5) * (1.0 / 4294967296.0);
+    e = -ln_pos(v);
+  }
+  return ln_pos(e);
+}
+
+// Exact race key in natural-log units, inv_T = 1 / T in double; greedy rows use -z.
+ERSD_HD double exact_key(uint32_t x, float z, double inv_T, bool greedy) {
   if (z != z) return (double)INFINITY;  // NaN logit counts as -inf
-  if (T == 0.0f) return -(double)z;
-  return exact_ln_e(x) - (double)z / (double)T;
+  if (greedy) return -(double)z;
+  if (z == INFINITY) return -(double)INFINITY;
+  if (z == -INFINITY) return (double)INFINITY;
+  return fma(-(double)z, inv_T, exact_ln_e(x));
+}
+ERSD_HD double exact_key(uint32_t x, float z, float T) {
+  return exact_key(x, z, T == 0.0f ? 0.0 : 1.0 / (double)T, T == 0.0f);
 }
 
 // Screening value: log2(e) in single precision from one int->float conversion

@@ -347,6 +347,22 @@ def test_screening_log_on_the_device_over_all_regimes(ersd):
     assert worst < 2.0**-11
 
 
+def test_deciding_logarithm_on_the_device(ersd):
+    """The straight-line double-precision ln(-log1p(-w)) that decides winners (hardware reciprocal
+    seed + Newton steps on the device) against the CUDA math library, over all regimes of x."""
+    V = 1 << 20
+    g = torch.Generator().manual_seed(12)
+    rows = [torch.zeros(V, dtype=torch.float32), wl.zipf_rows(1, V, g, "cpu")[0]]
+    out = torch.empty(V, dtype=torch.float32, device="cuda")
+    worst = 0.0
+    for row in rows:
+        for pos, T in ((0, 1.0), (1, 0.6), (2, 1.7)):
+            ersd.ersd_row_keys(row.cuda(), T, 99, 1, pos, 2, out)
+            torch.cuda.synchronize()
+            worst = max(worst, float(out.abs().max().item()))
+    assert worst < 0.05, worst          # units of 1e-12: below 5e-14
+
+
 def test_caller_owned_workspace_and_repeats(ersd):
     w = wl.scaled(wl.CONFIGS["c2"], B=3)
     inp = to_dev(wl.make_inputs(w, call=5))
