@@ -289,6 +289,15 @@ struct RoleInfo {
   int aligned;      // rows start on 16-byte boundaries
 };
 
+// What the block works on (written by thread 0 in setup_piece, read by everybody after it).
+struct Job {
+  int unit, b, r, s;   // logit row (b * rows + r), sequence, row in the sequence, chunk of the row
+  int cq, c0;          // children of the row's node (0: no draft row), arrivals wanted from the target row
+  int v0, v1;          // vocabulary range of the chunk
+  int valid_T;
+  float T, c2;         // temperature; keys are screened in log2 units: lg2(e) - z * c2
+};
+
 template <int DT>
 struct __align__(16) Shared {
   // streaming ring: [stage][role][vector][thread], filled by cp.async, each thread reading back
@@ -302,9 +311,19 @@ struct __align__(16) Shared {
   float tau[2];  // log2 units: no index whose true key exceeds tau[r] can be among the first c
   alignas(8) float lim[2];  // lim_of_tau(tau[r])
   int last;
+  Job job;
   int ttok[ERSD_MAX_ROWS], dtok[ERSD_MAX_ROWS];
   float tkey[ERSD_MAX_ROWS], dkey[ERSD_MAX_ROWS];
 };
+
+// The block's state lives at the start of dynamic shared memory; every function names it
+// through this accessor, so the compiler sees shared-space addresses (no generic loads) and no
+// pointer travels through the out-of-line calls.
+extern __shared__ __align__(16) unsigned char ersd_dyn_smem[];
+template <int DT>
+__device__ __forceinline__ Shared<DT>& block_state() {
+  return *reinterpret_cast<Shared<DT>*>(ersd_dyn_smem);
+}
 
 // After an insertion into warp `warp`'s list of role r: its c-th key bounds the role's threshold.
 template <int DT>
@@ -334,9 +353,8 @@ __device__ __forceinline__ float ring_logit(const Shared<DT>& sh, int stage, int
 // key and, if it is within the slack of the threshold, the double-precision key that decides;
 // survivors enter the warp's list.
 template <int DT>
-__device__ __noinline__ void settle_tile(Shared<DT>* shp, int stage, int i0, unsigned bits, float c2,
-                                         float T) {
-  Shared<DT>& sh = *shp;
+__device__ __noinline__ void settle_tile(int stage, int i0, unsigned bits, float c2, float T) {
+  Shared<DT>& sh = block_state<DT>();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const bool greedy = (T == 0.0f);
   __syncwarp();  // every lane's ring slot is complete and visible to the warp
@@ -387,8 +405,8 @@ __device__ __noinline__ void settle_tile(Shared<DT>* shp, int stage, int i0, uns
 // threshold goes to settle_tile, which finds the logits in ring stage `stage` (free at these
 // moments: the streaming loop has no copy in flight into it).
 template <int DT, int NR>
-__device__ __noinline__ void edge_tile(Shared<DT>* shp, int stage, int i0, int vend, float c2, float T) {
-  Shared<DT>& sh = *shp;
+__device__ __noinline__ void edge_tile(int stage, int i0, int vend, float c2, float T) {
+  Shared<DT>& sh = block_state<DT>();
   const int lane = threadIdx.x & 31;
   const bool greedy = (T == 0.0f);
   Raw<DT> raw[NR];
@@ -422,7 +440,7 @@ __device__ __noinline__ void edge_tile(Shared<DT>* shp, int stage, int i0, int v
     if (m <= tau + screen_slack(tau)) bits |= 1u << r;
   }
   __syncwarp();
-  if (__any_sync(kFull, bits != 0)) settle_tile<DT>(shp, stage, i0, bits, c2, T);
+  if (__any_sync(kFull, bits != 0)) settle_tile<DT>(stage, i0, bits, c2, T);
 }
 
 // The streaming loop over `ntiles` full tiles of 16-byte aligned rows; the thread's first index is
@@ -457,7 +475,8 @@ struct Streamer {
   }
 
   // Requests the first kStages - 1 tiles; call before any other work so the copies overlap it.
-  __device__ __forceinline__ void begin(Shared<DT>* sh, int i0, int ntiles_) {
+  __device__ __forceinline__ void begin(int i0, int ntiles_) {
+    Shared<DT>* sh = &block_state<DT>();
     ntiles = ntiles_;
     requested = 0;
     const uint32_t ring0 = (uint32_t)__cvta_generic_to_shared(&sh->ring[0][0][0][threadIdx.x]);
@@ -467,38 +486,49 @@ struct Streamer {
     for (int s = 0; s < kStages - 1; ++s) request_one(ring0);
   }
 
-  __device__ __forceinline__ void run(Shared<DT>* sh, int i0, float c2, float T) {
+  __device__ __forceinline__ void run(int i0, float c2, float T) {
+    Shared<DT>* sh = &block_state<DT>();
     const bool greedy = (T == 0.0f);
     const PhiloxRow pr = sh->philox;
     const uint32_t ring0 = (uint32_t)__cvta_generic_to_shared(&sh->ring[0][0][0][threadIdx.x]);
     const uint32_t lim_addr = (uint32_t)__cvta_generic_to_shared(sh->lim);
-    for (int t = 0; t < ntiles; ++t) {
-      request_one(ring0);
-      cp_async_wait<kStages - 1>();
-      const int stage = t % kStages;
-      float zub[NR];
-#pragma unroll
-      for (int r = 0; r < NR; ++r) {
-        Raw<DT> cur;
-#pragma unroll
-        for (int v = 0; v < kVec; ++v) cur.v[v] = sh->ring[stage][r][v][threadIdx.x];
-        zub[r] = logits_upper_bound(cur);
-      }
-      uint32_t xs[8];
-      pr.words((uint32_t)i0 >> 2, xs);
-      pr.words(((uint32_t)i0 >> 2) + 1u, xs + 4);
-      const uint32_t xm = min(__vimin3_u32(xs[0], xs[1], xs[2]),
-                              __vimin3_u32(__vimin3_u32(xs[3], xs[4], xs[5]), xs[6], xs[7]));
-      const float lgm = greedy ? 32.0f : lg2_fast((float)xm);
-      float2 lim;  // both roles' comparison values in one volatile load
-      asm volatile("ld.volatile.shared.v2.f32 {%0,%1}, [%2];" : "=f"(lim.x), "=f"(lim.y) : "r"(lim_addr));
+    int t = 0;
+    while (t < ntiles) {
+      // inner loop: no call inside, left only when some lane cannot rule its indices out
       unsigned bits = 0;
-      if (!(fmaf(-zub[0], c2, lgm) > lim.x)) bits |= 1u;
-      if (NR == 2) {
-        if (!(fmaf(-zub[NR - 1], c2, lgm) > lim.y)) bits |= 2u;
+      int stage = 0;
+      for (; t < ntiles; ++t, i0 += kTile) {
+        request_one(ring0);
+        cp_async_wait<kStages - 1>();
+        stage = t % kStages;
+        float zub[NR];
+#pragma unroll
+        for (int r = 0; r < NR; ++r) {
+          Raw<DT> cur;
+#pragma unroll
+          for (int v = 0; v < kVec; ++v) cur.v[v] = sh->ring[stage][r][v][threadIdx.x];
+          zub[r] = logits_upper_bound(cur);
+        }
+        uint32_t xs[8];
+        pr.words((uint32_t)i0 >> 2, xs);
+        pr.words(((uint32_t)i0 >> 2) + 1u, xs + 4);
+        const uint32_t xm = min(__vimin3_u32(xs[0], xs[1], xs[2]),
+                                __vimin3_u32(__vimin3_u32(xs[3], xs[4], xs[5]), xs[6], xs[7]));
+        const float lgm = greedy ? 32.0f : lg2_fast((float)xm);
+        float2 lim;  // both roles' comparison values in one volatile load
+        asm volatile("ld.volatile.shared.v2.f32 {%0,%1}, [%2];" : "=f"(lim.x), "=f"(lim.y) : "r"(lim_addr));
+        bits = 0;
+        if (!(fmaf(-zub[0], c2, lgm) > lim.x)) bits |= 1u;
+        if (NR == 2) {
+          if (!(fmaf(-zub[NR - 1], c2, lgm) > lim.y)) bits |= 2u;
+        }
+        if (__any_sync(kFull, bits != 0)) break;
       }
-      if (__any_sync(kFull, bits != 0)) settle_tile<DT>(sh, stage, i0, bits, c2, T);
-      i0 += kTile;
+      if (t < ntiles) {
+        settle_tile<DT>(stage, i0, bits, c2, T);
+        ++t;
+        i0 += kTile;
+      }
     }
   }
 };
@@ -507,8 +537,11 @@ struct Streamer {
 // the piece starts with a threshold for every role (handed down by an earlier piece of the same
 // row) all full tiles go through the streaming loop; otherwise the first tile is looked at index
 // by index to produce one.
+// (Inlined into the kernel, whose other parts are out-of-line calls: the loop then gets a
+// register allocation of its own.)
 template <int DT, int NR>
-__device__ __noinline__ void stream_piece(Shared<DT>* sh, int v0, int v1, float c2, float T) {
+__device__ __forceinline__ void stream_piece(int v0, int v1, float c2, float T) {
+  Shared<DT>* sh = &block_state<DT>();
   constexpr int kStages = Geo<DT>::kStages;
   const int tid = threadIdx.x;
   bool ring_ok = true, have_tau = true;
@@ -523,15 +556,15 @@ __device__ __noinline__ void stream_piece(Shared<DT>* sh, int v0, int v1, float 
   if (ring_ok) {
     const int first = have_tau ? 0 : 1;      // first tile of the streaming loop
     Streamer<DT, NR> st;
-    st.begin(sh, i0 + first * kTile, nfull > first ? nfull - first : 0);
+    st.begin(i0 + first * kTile, nfull > first ? nfull - first : 0);
     // no threshold yet: the first tile yields one (the requests above leave the last stage free)
-    if (!have_tau) edge_tile<DT, NR>(sh, kStages - 1, i0, v1, c2, T);
-    if (nfull > first) st.run(sh, i0 + first * kTile, c2, T);
+    if (!have_tau) edge_tile<DT, NR>(kStages - 1, i0, v1, c2, T);
+    if (nfull > first) st.run(i0 + first * kTile, c2, T);
     cp_async_wait<0>();
     if (ntiles > nfull && (have_tau || ntiles > 1))
-      edge_tile<DT, NR>(sh, 0, i0 + (ntiles - 1) * kTile, v1, c2, T);
+      edge_tile<DT, NR>(0, i0 + (ntiles - 1) * kTile, v1, c2, T);
   } else {
-    for (int t = 0; t < ntiles; ++t, i0 += kTile) edge_tile<DT, NR>(sh, 0, i0, v1, c2, T);
+    for (int t = 0; t < ntiles; ++t, i0 += kTile) edge_tile<DT, NR>(0, i0, v1, c2, T);
   }
 }
 
@@ -547,36 +580,35 @@ __device__ __forceinline__ void merge_partials(WarpList& L, const Entry* part, i
   }
 }
 
+// Decodes the block's work item and prepares the shared state.  Work items are ordered
+// chunk-major: every row's first chunk is scheduled before any second chunk, so that later
+// chunks of a row usually start with the threshold an earlier one left in the workspace;
+// within a chunk index rows follow tree.order (the heavier paired rows first).
 template <int DT>
-__global__ void __launch_bounds__(kThreads, ERSD_MIN_BLOCKS)
-ersd_race_kernel(const Params p, const __grid_constant__ TreeDesc tree) {
-  __shared__ Shared<DT> sh;
-
+__device__ __noinline__ void setup_piece(const Params& p, const TreeDesc& tree) {
+  Shared<DT>& sh = block_state<DT>();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  // work item -> (chunk, row, sequence), chunk-major: every row's first chunk is scheduled
-  // before any second chunk, so that later chunks of a row usually start with the threshold
-  // an earlier one left in the workspace; within a chunk index rows follow tree.order (the
-  // heavier paired rows first)
-  const int n_units = p.B * p.rows;
-  const int s = blockIdx.x / n_units;
-  const int rem = blockIdx.x - s * n_units;
-  const int ri = rem / p.B;
-  const int b = rem - ri * p.B;
-  const int r = (p.mode == kSample) ? ri : (int)tree.order[ri];
-  const int unit = b * p.rows + r;
-
-  const int cq = (p.mode == kSample) ? 0 : (int)tree.nchild[r];
-  const int c0 = (p.mode == kSample) ? p.c_sample : 1;
-  const int v0 = s * p.per_chunk;
-  const int v1 = min(p.V, v0 + p.per_chunk);
-
-  const float T = p.temps ? p.temps[(int64_t)b * p.ts_b + (int64_t)r * p.ts_r] : p.T;
-  const bool valid_T = (T >= 0.0f && T < INFINITY);
-  // keys are screened in log2 units: lg2(e) - z * c2 (greedy rows: -z * log2(e), no race)
-  const float c2 = (T == 0.0f) ? kLog2e : (float)(1.4426950408889634 / (double)T);
-
-  const size_t es = (DT == ERSD_BF16) ? 2 : 4;
   if (tid == 0) {
+    const int n_units = p.B * p.rows;
+    const int s = blockIdx.x / n_units;
+    const int rem = blockIdx.x - s * n_units;
+    const int ri = rem / p.B;
+    const int b = rem - ri * p.B;
+    const int r = (p.mode == kSample) ? ri : (int)tree.order[ri];
+    const int unit = b * p.rows + r;
+    const int cq = (p.mode == kSample) ? 0 : (int)tree.nchild[r];
+    const int c0 = (p.mode == kSample) ? p.c_sample : 1;
+    const float T = p.temps ? p.temps[(int64_t)b * p.ts_b + (int64_t)r * p.ts_r] : p.T;
+    Job j;
+    j.unit = unit; j.b = b; j.r = r; j.s = s; j.cq = cq; j.c0 = c0;
+    j.v0 = s * p.per_chunk;
+    j.v1 = min(p.V, j.v0 + p.per_chunk);
+    j.valid_T = (T >= 0.0f && T < INFINITY);
+    j.T = T;
+    j.c2 = (T == 0.0f) ? kLog2e : (float)(1.4426950408889634 / (double)T);  // greedy: -z log2(e)
+    sh.job = j;
+
+    const size_t es = (DT == ERSD_BF16) ? 2 : 4;
     const uint64_t seed = p.seeds[b];
     const uint32_t seq = p.seq_ids ? p.seq_ids[b] : (uint32_t)b;
     const uint32_t pos = (p.pos_offsets ? p.pos_offsets[b] : 0u) + (uint32_t)r;
@@ -597,22 +629,23 @@ ersd_race_kernel(const Params p, const __grid_constant__ TreeDesc tree) {
       sh.lim[q] = (tau < INFINITY) ? lim_of_tau(tau) : INFINITY;
     }
   }
-  {
-    Entry e;
-    e.key = (double)INFINITY;
-    e.idx = 0x7FFFFFFF;
-    e.pad = 0;
-    sh.list[0][warp][lane] = e;
-    sh.list[1][warp][lane] = e;
-  }
+  Entry e;
+  e.key = (double)INFINITY;
+  e.idx = 0x7FFFFFFF;
+  e.pad = 0;
+  sh.list[0][warp][lane] = e;
+  sh.list[1][warp][lane] = e;
   __syncthreads();
+}
 
-  if (valid_T) {  // a row with an invalid temperature has no arrivals
-    if (cq > 0) stream_piece<DT, 2>(&sh, v0, v1, c2, T);
-    else stream_piece<DT, 1>(&sh, v0, v1, c2, T);
-  }
-  __syncthreads();
-
+// After the streaming: merges the warps' lists, hands the chunk's arrivals to the workspace and,
+// in the block that completes the group (row in sample mode, sequence otherwise), turns the
+// winners into the call's outputs.
+template <int DT>
+__device__ __noinline__ void finish_piece(const Params& p, const TreeDesc& tree) {
+  Shared<DT>& sh = block_state<DT>();
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int unit = sh.job.unit, b = sh.job.b, s = sh.job.s, cq = sh.job.cq, c0 = sh.job.c0;
   // ---- block merge: warp `role` merges the eight warps' lists of that role ----
   const int nroles = cq > 0 ? 2 : 1;
   const bool direct = (p.mode == kSample && p.S == 1);
@@ -755,6 +788,21 @@ ersd_race_kernel(const Params p, const __grid_constant__ TreeDesc tree) {
     }
     p.out_accept_len[b] = depth;
   }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads, ERSD_MIN_BLOCKS)
+ersd_race_kernel(const __grid_constant__ Params p, const __grid_constant__ TreeDesc tree) {
+  setup_piece<DT>(p, tree);
+  {
+    const Job& j = block_state<DT>().job;
+    if (j.valid_T) {  // a row with an invalid temperature has no arrivals
+      if (j.cq > 0) stream_piece<DT, 2>(j.v0, j.v1, j.c2, j.T);
+      else stream_piece<DT, 1>(j.v0, j.v1, j.c2, j.T);
+    }
+  }
+  __syncthreads();
+  finish_piece<DT>(p, tree);
 }
 
 template <int DT>
@@ -946,6 +994,12 @@ static int prefer_shared_memory() {
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(ersd_race_kernel<ERSD_F32>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                cudaSharedmemCarveoutMaxShared);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(ersd_race_kernel<ERSD_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)sizeof(Shared<ERSD_BF16>));
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(ersd_race_kernel<ERSD_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)sizeof(Shared<ERSD_F32>));
     if (e != cudaSuccess) return cuda_fail(e);
     done[dev] = true;
   }
@@ -957,8 +1011,8 @@ static int launch(const Params& p, const TreeDesc& tree, int dt, cudaStream_t st
   if (items > 0x7FFFFFFF) return ERSD_EINVAL;
   const int pst = prefer_shared_memory();
   if (pst != ERSD_OK) return pst;
-  if (dt == ERSD_BF16) ersd_race_kernel<ERSD_BF16><<<(unsigned)items, kThreads, 0, st>>>(p, tree);
-  else ersd_race_kernel<ERSD_F32><<<(unsigned)items, kThreads, 0, st>>>(p, tree);
+  if (dt == ERSD_BF16) ersd_race_kernel<ERSD_BF16><<<(unsigned)items, kThreads, sizeof(Shared<ERSD_BF16>), st>>>(p, tree);
+  else ersd_race_kernel<ERSD_F32><<<(unsigned)items, kThreads, sizeof(Shared<ERSD_F32>), st>>>(p, tree);
   const cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? ERSD_OK : cuda_fail(e);
 }
