@@ -475,13 +475,13 @@ struct Streamer {
   }
 
   // Requests the first kStages - 1 tiles; call before any other work so the copies overlap it.
-  __device__ __forceinline__ void begin(int i0, int ntiles_) {
+  __device__ __forceinline__ void begin(const char* const* rows, int i0, int ntiles_) {
     Shared<DT>* sh = &block_state<DT>();
     ntiles = ntiles_;
     requested = 0;
     const uint32_t ring0 = (uint32_t)__cvta_generic_to_shared(&sh->ring[0][0][0][threadIdx.x]);
 #pragma unroll
-    for (int r = 0; r < NR; ++r) src[r] = sh->role[r].row + (size_t)i0 * kElem;
+    for (int r = 0; r < NR; ++r) src[r] = rows[r] + (size_t)i0 * kElem;
 #pragma unroll
     for (int s = 0; s < kStages - 1; ++s) request_one(ring0);
   }
@@ -533,36 +533,62 @@ struct Streamer {
   }
 };
 
-// One piece = chunk [v0, v1) of a logit row (NR = 1) or of a draft/target pair (NR = 2).  When
-// the piece starts with a threshold for every role (handed down by an earlier piece of the same
-// row) all full tiles go through the streaming loop; otherwise the first tile is looked at index
-// by index to produce one.
+// The first tile of a chunk that starts with a threshold for every role: the same cheap test as
+// in the streaming loop, on logits fetched with plain loads (and parked in ring stage `stage`
+// for settle_tile).
+template <int DT, int NR>
+__device__ __noinline__ void first_tile(int stage, int i0, int vend, float c2, float T) {
+  Shared<DT>& sh = block_state<DT>();
+  const bool greedy = (T == 0.0f);
+  float zub[NR];
+#pragma unroll
+  for (int r = 0; r < NR; ++r) {
+    const Raw<DT> raw = fetch<DT>(sh.role[r].row, i0, vend, true);
+#pragma unroll
+    for (int v = 0; v < Geo<DT>::kVec; ++v) sh.ring[stage][r][v][threadIdx.x] = raw.v[v];
+    zub[r] = logits_upper_bound(raw);
+  }
+  uint32_t xs[8];
+  sh.philox.words((uint32_t)i0 >> 2, xs);
+  sh.philox.words(((uint32_t)i0 >> 2) + 1u, xs + 4);
+  const uint32_t xm = min(__vimin3_u32(xs[0], xs[1], xs[2]),
+                          __vimin3_u32(__vimin3_u32(xs[3], xs[4], xs[5]), xs[6], xs[7]));
+  const float lgm = greedy ? 32.0f : lg2_fast((float)xm);
+  unsigned bits = 0;
+#pragma unroll
+  for (int r = 0; r < NR; ++r)
+    if (!(fmaf(-zub[r], c2, lgm) > *(volatile float*)&sh.lim[r])) bits |= 1u << r;
+  if (__any_sync(kFull, bits != 0)) settle_tile<DT>(stage, i0, bits, c2, T);
+}
+
+// One piece = chunk [v0, v1) of a logit row (NR = 1) or of a draft/target pair (NR = 2); rows[]
+// point at the rows' first elements.  The streaming loop takes the full tiles after the first
+// (its trip count depends only on launch parameters, which keeps the loop control on the
+// uniform datapath); the first tile yields the first threshold unless an earlier chunk of the
+// row handed one down; a ragged last tile is looked at index by index.
 // (Inlined into the kernel, whose other parts are out-of-line calls: the loop then gets a
 // register allocation of its own.)
 template <int DT, int NR>
-__device__ __forceinline__ void stream_piece(int v0, int v1, float c2, float T) {
-  Shared<DT>* sh = &block_state<DT>();
+__device__ __forceinline__ void stream_piece(const char* const* rows, bool ring_ok, int v0, int v1,
+                                             float c2, float T) {
   constexpr int kStages = Geo<DT>::kStages;
+  Shared<DT>* sh = &block_state<DT>();
   const int tid = threadIdx.x;
-  bool ring_ok = true, have_tau = true;
-#pragma unroll
-  for (int r = 0; r < NR; ++r) {
-    ring_ok = ring_ok && (sh->role[r].aligned != 0);
-    have_tau = have_tau && (sh->tau[r] < INFINITY);
-  }
   const int ntiles = (v1 - v0 + kTile - 1) / kTile;
   const int nfull = (v1 - v0) / kTile;       // tiles that lie fully inside the piece
   int i0 = v0 + tid * kPerThread;
   if (ring_ok) {
-    const int first = have_tau ? 0 : 1;      // first tile of the streaming loop
     Streamer<DT, NR> st;
-    st.begin(i0 + first * kTile, nfull > first ? nfull - first : 0);
-    // no threshold yet: the first tile yields one (the requests above leave the last stage free)
-    if (!have_tau) edge_tile<DT, NR>(kStages - 1, i0, v1, c2, T);
-    if (nfull > first) st.run(i0 + first * kTile, c2, T);
+    st.begin(rows, i0 + kTile, nfull > 1 ? nfull - 1 : 0);
+    // (the requests above leave the last ring stage free for the first tile's logits)
+    bool have_tau = (nfull >= 1);
+#pragma unroll
+    for (int r = 0; r < NR; ++r) have_tau = have_tau && (sh->tau[r] < INFINITY);
+    if (have_tau) first_tile<DT, NR>(kStages - 1, i0, v1, c2, T);
+    else edge_tile<DT, NR>(kStages - 1, i0, v1, c2, T);
+    if (nfull > 1) st.run(i0 + kTile, c2, T);
     cp_async_wait<0>();
-    if (ntiles > nfull && (have_tau || ntiles > 1))
-      edge_tile<DT, NR>(0, i0 + (ntiles - 1) * kTile, v1, c2, T);
+    if (ntiles > nfull && ntiles > 1) edge_tile<DT, NR>(0, i0 + (ntiles - 1) * kTile, v1, c2, T);
   } else {
     for (int t = 0; t < ntiles; ++t, i0 += kTile) edge_tile<DT, NR>(0, i0, v1, c2, T);
   }
@@ -588,42 +614,46 @@ template <int DT>
 __device__ __noinline__ void setup_piece(const Params& p, const TreeDesc& tree) {
   Shared<DT>& sh = block_state<DT>();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) {
-    const int n_units = p.B * p.rows;
-    const int s = blockIdx.x / n_units;
-    const int rem = blockIdx.x - s * n_units;
-    const int ri = rem / p.B;
-    const int b = rem - ri * p.B;
-    const int r = (p.mode == kSample) ? ri : (int)tree.order[ri];
-    const int unit = b * p.rows + r;
-    const int cq = (p.mode == kSample) ? 0 : (int)tree.nchild[r];
-    const int c0 = (p.mode == kSample) ? p.c_sample : 1;
-    const float T = p.temps ? p.temps[(int64_t)b * p.ts_b + (int64_t)r * p.ts_r] : p.T;
-    Job j;
-    j.unit = unit; j.b = b; j.r = r; j.s = s; j.cq = cq; j.c0 = c0;
-    j.v0 = s * p.per_chunk;
-    j.v1 = min(p.V, j.v0 + p.per_chunk);
-    j.valid_T = (T >= 0.0f && T < INFINITY);
-    j.T = T;
-    j.c2 = (T == 0.0f) ? kLog2e : (float)(1.4426950408889634 / (double)T);  // greedy: -z log2(e)
-    sh.job = j;
-
-    const size_t es = (DT == ERSD_BF16) ? 2 : 4;
-    const uint64_t seed = p.seeds[b];
-    const uint32_t seq = p.seq_ids ? p.seq_ids[b] : (uint32_t)b;
-    const uint32_t pos = (p.pos_offsets ? p.pos_offsets[b] : 0u) + (uint32_t)r;
-    sh.philox.init(seed, seq, pos);
-    sh.inv_T = (T == 0.0f) ? 0.0 : 1.0 / (double)T;
-    sh.role[0].row = (const char*)p.target + (size_t)unit * (size_t)p.ld_t * es;
-    sh.role[0].c = c0;
-    sh.role[0].aligned = p.aligned_t;
-    sh.role[1].row = cq > 0 ? (const char*)p.draft + ((size_t)b * p.draft_rows + r) * (size_t)p.ld_d * es
-                            : nullptr;
-    sh.role[1].c = cq > 0 ? cq : 1;
-    sh.role[1].aligned = p.aligned_d;
-    // thresholds handed down by earlier chunks of this row (any of them is a valid bound)
-#pragma unroll
-    for (int q = 0; q < 2; ++q) {
+  // every thread decodes (cheap, no memory); single lanes of different warps then fill in the
+  // parts of the state side by side, so that their memory latencies overlap
+  const int n_units = p.B * p.rows;
+  const int s = blockIdx.x / n_units;
+  const int rem = blockIdx.x - s * n_units;
+  const int ri = rem / p.B;
+  const int b = rem - ri * p.B;
+  const int r = (p.mode == kSample) ? ri : (int)tree.order[ri];
+  const int unit = b * p.rows + r;
+  const int cq = (p.mode == kSample) ? 0 : (int)tree.nchild[r];
+  const int c0 = (p.mode == kSample) ? p.c_sample : 1;
+  if (lane == 0) {
+    if (warp == 0) {
+      const uint64_t seed = p.seeds[b];
+      const uint32_t seq = p.seq_ids ? p.seq_ids[b] : (uint32_t)b;
+      const uint32_t pos = (p.pos_offsets ? p.pos_offsets[b] : 0u) + (uint32_t)r;
+      sh.philox.init(seed, seq, pos);
+    } else if (warp == 1) {
+      const float T = p.temps ? p.temps[(int64_t)b * p.ts_b + (int64_t)r * p.ts_r] : p.T;
+      Job j;
+      j.unit = unit; j.b = b; j.r = r; j.s = s; j.cq = cq; j.c0 = c0;
+      j.v0 = s * p.per_chunk;
+      j.v1 = min(p.V, j.v0 + p.per_chunk);
+      j.valid_T = (T >= 0.0f && T < INFINITY);
+      j.T = T;
+      j.c2 = (T == 0.0f) ? kLog2e : (float)(1.4426950408889634 / (double)T);  // greedy: -z log2(e)
+      sh.job = j;
+      sh.inv_T = (T == 0.0f) ? 0.0 : 1.0 / (double)T;
+    } else if (warp == 2) {
+      const size_t es = (DT == ERSD_BF16) ? 2 : 4;
+      sh.role[0].row = (const char*)p.target + (size_t)unit * (size_t)p.ld_t * es;
+      sh.role[0].c = c0;
+      sh.role[0].aligned = p.aligned_t;
+      sh.role[1].row = cq > 0 ? (const char*)p.draft + ((size_t)b * p.draft_rows + r) * (size_t)p.ld_d * es
+                              : nullptr;
+      sh.role[1].c = cq > 0 ? cq : 1;
+      sh.role[1].aligned = p.aligned_d;
+    } else if (warp == 3 || warp == 4) {
+      // thresholds handed down by earlier chunks of this row (any of them is a valid bound)
+      const int q = warp - 3;
       const float tau = (p.S > 1) ? tau_of_code(__ldcg(&p.slots[unit].tau_code[q])) : INFINITY;
       sh.tau[q] = tau;
       sh.lim[q] = (tau < INFINITY) ? lim_of_tau(tau) : INFINITY;
@@ -653,13 +683,27 @@ __device__ __noinline__ void finish_piece(const Params& p, const TreeDesc& tree)
     const int role = warp;
     const int c = sh.role[role].c;
     WarpList L;
-    L.key = sh.list[role][0][lane].key;
-    L.idx = sh.list[role][0][lane].idx;
-    for (int w = 1; w < kWarps; ++w) {
-      for (int e = 0; e < c; ++e) {
-        const Entry en = sh.list[role][w][e];
-        if (en.idx == 0x7FFFFFFF) break;
-        L.insert(en.key, en.idx, lane);
+    if (c == 1) {  // winners only: lane w takes warp w's best, a shuffle tree finds the smallest
+      L.key = lane < kWarps ? sh.list[role][lane][0].key : (double)INFINITY;
+      L.idx = lane < kWarps ? sh.list[role][lane][0].idx : 0x7FFFFFFF;
+#pragma unroll
+      for (int off = kWarps / 2; off > 0; off >>= 1) {
+        const double ok = __shfl_down_sync(kFull, L.key, off);
+        const int oi = __shfl_down_sync(kFull, L.idx, off);
+        if (ok < L.key || (ok == L.key && oi < L.idx)) {
+          L.key = ok;
+          L.idx = oi;
+        }
+      }
+    } else {
+      L.key = sh.list[role][0][lane].key;
+      L.idx = sh.list[role][0][lane].idx;
+      for (int w = 1; w < kWarps; ++w) {
+        for (int e = 0; e < c; ++e) {
+          const Entry en = sh.list[role][w][e];
+          if (en.idx == 0x7FFFFFFF) break;
+          L.insert(en.key, en.idx, lane);
+        }
       }
     }
     if (direct) {
@@ -793,12 +837,29 @@ __device__ __noinline__ void finish_piece(const Params& p, const TreeDesc& tree)
 template <int DT>
 __global__ void __launch_bounds__(kThreads, ERSD_MIN_BLOCKS)
 ersd_race_kernel(const __grid_constant__ Params p, const __grid_constant__ TreeDesc tree) {
+  // The same decode as in setup_piece, from launch parameters only: everything here is uniform
+  // over the block, and the compiler can tell.
+  const int n_units = p.B * p.rows;
+  const int s = blockIdx.x / n_units;
+  const int rem = blockIdx.x - s * n_units;
+  const int ri = rem / p.B;
+  const int b = rem - ri * p.B;
+  const int r = (p.mode == kSample) ? ri : (int)tree.order[ri];
+  const int cq = (p.mode == kSample) ? 0 : (int)tree.nchild[r];
+  const int v0 = s * p.per_chunk;
+  const int v1 = min(p.V, v0 + p.per_chunk);
+  const size_t es = (DT == ERSD_BF16) ? 2 : 4;
+  const char* rows[2];
+  rows[0] = (const char*)p.target + ((size_t)b * p.rows + r) * (size_t)p.ld_t * es;
+  rows[1] = (const char*)p.draft + ((size_t)b * p.draft_rows + r) * (size_t)p.ld_d * es;
+  const bool ring_ok = p.aligned_t && (cq == 0 || p.aligned_d);
+
   setup_piece<DT>(p, tree);
   {
     const Job& j = block_state<DT>().job;
     if (j.valid_T) {  // a row with an invalid temperature has no arrivals
-      if (j.cq > 0) stream_piece<DT, 2>(j.v0, j.v1, j.c2, j.T);
-      else stream_piece<DT, 1>(j.v0, j.v1, j.c2, j.T);
+      if (cq > 0) stream_piece<DT, 2>(rows, ring_ok, v0, v1, j.c2, j.T);
+      else stream_piece<DT, 1>(rows, ring_ok, v0, v1, j.c2, j.T);
     }
   }
   __syncthreads();
