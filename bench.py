@@ -30,6 +30,12 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# profiles/: dram bytes (read + write) per algorithmic byte of one launch, and the library version
+# the counters were taken at
+DRAM_BYTES_PER_ALGORITHMIC_BYTE = 1.012
+TRAFFIC_AT_VERSION = 101
+SM_COUNT = 148
+
 METRIC = "race-verified logit rows/s at V=128256 bf16 (B*(k+1) rows)"
 UNIT = "rows/s"
 
@@ -174,7 +180,8 @@ def main():
     ap.add_argument("--sets", type=int, default=3, help="distinct input sets rotated between launches")
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--ref-seqs", type=int, default=64, help="sequences per oracle step (reference arm)")
-    ap.add_argument("--cpu-seqs", type=int, default=96, help="sequences of the oracle sample (cpu_baseline)")
+    ap.add_argument("--cpu-seqs", type=int, default=0, help="sequences of the oracle sample (cpu_baseline); 0 = all")
+    ap.add_argument("--cpu-passes", type=int, default=8, help="passes of the oracle over its sample (cpu_baseline)")
     ap.add_argument("--split", type=int, default=0, help="thread blocks per row (0: library default)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -243,6 +250,8 @@ def main():
     time.sleep(0.25)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    # profiler range = the timed region (a no-op unless a profiler asked for --profile-from-start off)
+    torch.cuda.cudart().cudaProfilerStart()
     t_wall0 = time.time()
     ev0.record(stream)
     for i in range(args.steps):
@@ -250,6 +259,7 @@ def main():
     ev1.record(stream)
     barrier()
     t_wall1 = time.time()
+    torch.cuda.cudart().cudaProfilerStop()
     clocks = sampler.stop(t_wall0, t_wall1)
     ms_total = ev0.elapsed_time(ev1)
     if dist is not None:
@@ -265,16 +275,21 @@ def main():
     peak, peak_kind = load_peaks()
     alg_bytes = algorithmic_bytes(w, sets[0])
     achieved = alg_bytes / (ms_step * 1e-3) / 1e9
+    # DRAM traffic per launch from the ncu capture summarised in profiles/ (dram read + write bytes
+    # over algorithmic bytes, taken on this workload); void once the kernel has changed since
     traffic = None
-    tpath = os.path.join(ROOT, "profiles", "traffic_per_index.json")
-    if os.path.exists(tpath):
-        with open(tpath) as f:
-            tj = json.load(f)
-        traffic = tj["dram_bytes_per_algorithmic_byte"] * alg_bytes
+    if binding.ersd_version() == TRAFFIC_AT_VERSION:
+        traffic = DRAM_BYTES_PER_ALGORITHMIC_BYTE * alg_bytes
+    # the other roof: every vocabulary index needs a quarter of a Philox4x32-10 call, 4.5 wide
+    # multiplies and 4.75 three-input xors on the integer path (64 lanes per clock and SM)
+    n_index = w.B * w.rows_target * w.V
+    t_alu_ms = n_index * 9.25 / (64.0 * SM_COUNT * (clocks["sm_max_mhz"] or 1965.0) * 1e6) * 1e3
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": traffic, "peak_kind": peak_kind + " copy bandwidth",
                 "algorithmic_bytes_per_launch": alg_bytes, "kernel": "ersd_race_kernel<bf16>",
-                "kernel_ms": ms_step}
+                "kernel_ms": ms_step, "t_hbm_ms": alg_bytes / (peak * 1e9) * 1e3,
+                "t_int_ms": t_alu_ms,
+                "note": "t_int_ms: Philox integer work alone at the nominal 64 int lanes/clk/SM"}
 
     # ---- end to end: host buffers in pinned memory, copies inside the timed region
     e2e = None
@@ -307,11 +322,16 @@ def main():
     # ---- the oracle on the host cores, on a bounded sample of the same workload (rank 0, N = 1)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        n_seq = max(1, min(w.B, args.cpu_seqs))
-        rate, secs, cores = oracle_rate(w, sets[0], n_seq)
+        n_seq = w.B if args.cpu_seqs <= 0 else max(1, min(w.B, args.cpu_seqs))
+        t_cpu0 = time.perf_counter()
+        rates = [oracle_rate(w, sets[0], n_seq) for _ in range(max(1, args.cpu_passes))]
+        t_cpu = time.perf_counter() - t_cpu0
+        rate = statistics.median(r[0] for r in rates)
+        cores = rates[0][2]
         cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": "first %d of %d sequences of input set 0 (%d logit rows), one pass, %.2f s" % (
-                   n_seq, w.B, n_seq * (w.rows_target + w.k), secs)}
+               "sample": "first %d of %d sequences of input set 0 (%d logit rows), median of %d passes, "
+                         "%.1f s of wall time in all" % (n_seq, w.B, n_seq * (w.rows_target + w.k),
+                                                         len(rates), t_cpu)}
 
     if rank == 0:
         print(json.dumps({
