@@ -64,7 +64,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -173,7 +173,7 @@ def workload_config(w, l2_note):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="c5")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -197,7 +197,7 @@ def main():
         return
 
     import torch
-    from paper_2504_15475_b200 import binding
+    from paper_2504_15475_b200 import binding, replicas
     binding.lib()  # fail loudly if the CUDA library is missing
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -213,7 +213,7 @@ def main():
     # ---- inputs: resident in HBM before the timed region; every rank has its own replica
     sets = []
     for s in range(max(1, args.sets)):
-        sets.append(wl.make_inputs(w, call=rank * 100 + s, device="cuda", sigma=args.sigma,
+        sets.append(wl.make_inputs(w, call=replicas.replica_call_index(rank, s), device="cuda", sigma=args.sigma,
                                    T=args.temperature))
     D = w.k if not w.is_tree else binding.ersd_tree_depth(w.parent)
     tokens = torch.empty(w.B, D + 1, dtype=torch.int32, device="cuda")
@@ -261,14 +261,8 @@ def main():
     t_wall1 = time.time()
     torch.cuda.cudart().cudaProfilerStop()
     clocks = sampler.stop(t_wall0, t_wall1)
-    ms_total = ev0.elapsed_time(ev1)
-    if dist is not None:
-        t = torch.tensor([ms_total], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
-    ms_step = ms_total / args.steps
     rows_per_step = w.B * w.rows_target
-    value = world * rows_per_step / (ms_step * 1e-3)
+    value, ms_step = replicas.whole_job_rate(rows_per_step, args.steps, ev0.elapsed_time(ev1), dist, "cuda")
     mean_accept = float(accept.float().mean().item())
 
     # ---- roofline of the one kernel a step launches
@@ -308,10 +302,7 @@ def main():
                                                parent=h.get("parent"))
         torch.cuda.synchronize()
         dt = (time.perf_counter() - t0) / args.e2e_steps
-        if dist is not None:
-            t = torch.tensor([dt], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
+        dt = replicas.max_over_ranks(dt, dist, "cuda")
         h2d = sum(x.numel() * x.element_size() for x in (host_t, host_d, host_s) if x is not None)
         if host_temps is not None:
             h2d += host_temps.numel() * 4
