@@ -965,16 +965,14 @@ static bool rows_aligned(const void* base, int64_t ld, int dt) {
   return ((uintptr_t)base & 15) == 0 && ((ld * elem_size(dt)) & 15) == 0;
 }
 
-#ifndef ERSD_WAVES
-#define ERSD_WAVES 3            // work items per resident-block slot that the default split aims for
-#endif
 #ifndef ERSD_MIN_CHUNK_TILES
 #define ERSD_MIN_CHUNK_TILES 8  // smallest chunk of a row that the default split makes
 #endif
 
-// Thread blocks per row.  Many more work items than resident blocks, so that the hardware's
-// block scheduler evens out rows of different cost and the last wave is short; chunks stay long
-// enough to amortise a block's set-up and merge.
+// Thread blocks per row.  At least one work item per resident-block slot, and two chunks per
+// row when rows are long: the hardware's block scheduler then evens out rows of different cost
+// and the last wave is made of half rows.  More chunks do not pay: each costs a block about as
+// much set-up, barrier and merge time as eight tiles of streaming (measured).
 static int choose_split(const ersd_opts& o, int64_t units, int V, int cmax) {
   int smax = kPartCap / cmax;
   if (smax > ERSD_MAX_SPLIT) smax = ERSD_MAX_SPLIT;
@@ -986,7 +984,8 @@ static int choose_split(const ersd_opts& o, int64_t units, int V, int cmax) {
     if (S > ntiles) S = ntiles;
   } else {
     const int64_t slots = 148 * ERSD_MIN_BLOCKS;
-    S = (int)((ERSD_WAVES * slots + units - 1) / units);
+    S = (int)((slots + units - 1) / units);
+    if (S < 2 && ntiles >= 4 * ERSD_MIN_CHUNK_TILES) S = 2;
     const int by_v = ntiles / ERSD_MIN_CHUNK_TILES;
     if (S > by_v) S = by_v;
   }
