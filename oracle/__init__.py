@@ -187,6 +187,36 @@ def verify(target: np.ndarray, draft: np.ndarray, seeds, T: float = 1.0, temps=N
     return out
 
 
+def verify_tokens(target: np.ndarray, draft_tokens: np.ndarray, seeds, T: float = 1.0, temps=None,
+                  seq_ids=None, pos_offsets=None):
+    """Verification when the drafted tokens are given (Algorithm 2's verification lines, extended
+    to a drafted sequence as Section 3 describes: accept in order until the first rejection).
+
+    target [B, k+1, V]; draft_tokens [B, k] (token drafted at position j, i.e. the draft row's race
+    winner under the SAME race variables, produced earlier).  Position j's target winner is
+    argmin_i e_i / p_i with that position's race; position j is accepted iff it equals
+    draft_tokens[b, j]; the output is the target winners up to and including the first
+    rejection (or the extra token of position k when all k are accepted).
+    Returns dict(tokens [B, k+1] (-1 padded), accept_len [B], target_tok, target_key [B, k+1, 2]).
+    """
+    target = np.ascontiguousarray(target)
+    B, rows, V = target.shape
+    k = rows - 1
+    draft_tokens = np.asarray(draft_tokens)
+    assert draft_tokens.shape == (B, k)
+    tok, key = race_sample(target, seeds, T=T, c=1, temps=temps, seq_ids=seq_ids, pos_offsets=pos_offsets)
+    ttok = tok[..., 0]
+    tokens = np.full((B, rows), -1, np.int32)
+    accept = np.zeros(B, np.int32)
+    for b in range(B):
+        L = 0
+        while L < k and ttok[b, L] >= 0 and ttok[b, L] == draft_tokens[b, L]:
+            L += 1
+        tokens[b, :L + 1] = ttok[b, :L + 1]
+        accept[b] = L
+    return dict(tokens=tokens, accept_len=accept, target_tok=ttok.astype(np.int32), target_key=key)
+
+
 def tree_shape(parent):
     """(depth D, max children, children counts, sibling ranks) of a parent array."""
     parent = np.asarray(parent, dtype=np.int64)

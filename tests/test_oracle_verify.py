@@ -204,3 +204,42 @@ def test_workload_recipe_shapes():
     assert set(np.unique(c5["temps"].numpy()).astype(np.float64).round(3).tolist()) <= {0.6, 0.8, 1.0}
     c1 = wl.make_inputs(wl.CONFIGS["c1"])
     assert c1["seeds"].tolist() == [0] and c1["target"].dtype == __import__("torch").float32
+
+
+def test_token_given_verification_agrees_with_the_row_given_one():
+    """Drafting first (winners of the draft rows) and then verifying the given tokens is the
+    sequence procedure of Section 3 cut in two: same accepted prefix, same emitted tokens."""
+    rng = np.random.default_rng(11)
+    B, k, V = 40, 5, 300
+    tgt = rng.normal(size=(B, k + 1, V)).astype(np.float32) * 2
+    drf = (tgt[:, :k] + rng.normal(size=(B, k, V)).astype(np.float32) * 0.7).astype(np.float32)
+    seeds = rng.integers(0, 2**63, size=B).astype(np.uint64)
+    full = oracle.verify(tgt, drf, seeds, T=0.9)
+    drafted, _ = oracle.race_sample(drf, seeds, T=0.9)
+    got = oracle.verify_tokens(tgt, drafted[..., 0], seeds, T=0.9)
+    assert (drafted[..., 0] == full["draft_tok"]).all()
+    assert (got["accept_len"] == full["accept_len"]).all()
+    assert (got["tokens"] == full["tokens"]).all()
+    assert 0 < got["accept_len"].mean() < k                   # both outcomes occur
+
+
+def test_token_given_verification_outcomes_of_algorithm_2():
+    """k = 1: a drafted token equal to the target winner gives two tokens, any other gives the
+    target winner alone; a wrong later token cuts the prefix exactly there."""
+    rng = np.random.default_rng(12)
+    B, V = 30, 50
+    tgt = rng.normal(size=(B, 2, V)).astype(np.float32)
+    seeds = np.arange(B, dtype=np.uint64) + 5
+    win, _ = oracle.race_sample(tgt, seeds, T=1.0)
+    hit = oracle.verify_tokens(tgt, win[:, :1, 0], seeds, T=1.0)
+    assert (hit["accept_len"] == 1).all() and (hit["tokens"] == win[..., 0]).all()
+    miss = oracle.verify_tokens(tgt, (win[:, :1, 0] + 1) % V, seeds, T=1.0)
+    assert (miss["accept_len"] == 0).all()
+    assert (miss["tokens"][:, 0] == win[:, 0, 0]).all() and (miss["tokens"][:, 1] == -1).all()
+    tgt3 = rng.normal(size=(B, 4, V)).astype(np.float32)
+    w3, _ = oracle.race_sample(tgt3, seeds, T=1.0)
+    d = w3[:, :3, 0].copy()
+    d[:, 1] = (d[:, 1] + 3) % V                               # second drafted token wrong
+    cut = oracle.verify_tokens(tgt3, d, seeds, T=1.0)
+    assert (cut["accept_len"] == 1).all() and (cut["tokens"][:, 2:] == -1).all()
+    assert (cut["tokens"][:, :2] == w3[:, :2, 0]).all()
