@@ -161,6 +161,26 @@ int ersd_verify_tree(const void* target_logits, const void* draft_logits, ersd_d
                      void* cuda_stream);
 
 /*
+ * Verification of tokens drafted earlier (Algorithm 2's verification lines on a
+ * drafted sequence, Section 3: accept in order until the first rejection).
+ * In a decoding loop the draft tokens already exist when the target model has
+ * run -- they were produced one position at a time with ersd_race_sample on
+ * the draft model's rows -- so only the target rows need to be raced:
+ * half the bytes of ersd_verify, same result as long as the tokens were
+ * drafted with the same (seed, sequence id, position) races.
+ *   target_logits device [B, k+1, V]      draft_tokens device [B, k] int32
+ *   out_tokens    device [B, k+1] int32   out_accept_len device [B] int32
+ * Position j < k is accepted iff its target winner equals draft_tokens[b, j];
+ * outputs as for ersd_verify.  opts->out_target_tok / out_target_key are
+ * filled if given; opts->out_draft_tok echoes draft_tokens, out_draft_key is
+ * filled with +inf.
+ * Errors as for ersd_verify (draft_tokens may be NULL only when k == 0).
+ */
+int ersd_verify_tokens(const void* target_logits, const int32_t* draft_tokens, ersd_dtype dt,
+                       const uint64_t* seeds, int B, int k, int V, float T, int32_t* out_tokens,
+                       int32_t* out_accept_len, const ersd_opts* opts, void* cuda_stream);
+
+/*
  * ersd_verify for callers that must not allocate device memory.  (The paper has
  * no counterpart; this is a deployment variant of ersd_verify and computes
  * exactly the same outputs from the same arguments.)

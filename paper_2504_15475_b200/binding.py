@@ -22,7 +22,7 @@ ERSD_MAX_TOP_C, ERSD_MAX_ROWS, ERSD_MAX_SPLIT = 32, 256, 32
 ERSD_NOALLOC_MAX_ROWS = 1024
 ERSD_ENOALLOC_LIMIT = -6
 
-EXPORTS = ("ersd_race_sample", "ersd_verify", "ersd_verify_noalloc", "ersd_verify_tree", "ersd_tree_depth",
+EXPORTS = ("ersd_race_sample", "ersd_verify", "ersd_verify_tokens", "ersd_verify_noalloc", "ersd_verify_tree", "ersd_tree_depth",
            "ersd_row_keys", "ersd_workspace_bytes", "ersd_workspace_init", "ersd_status_string",
            "ersd_last_cuda_error", "ersd_version")
 
@@ -65,6 +65,7 @@ def lib():
         L.ersd_race_sample.argtypes = [vp, i, vp, i, i, i, f, vp, C.POINTER(ErsdOpts), vp]
         L.ersd_verify.argtypes = [vp, vp, i, vp, i, i, i, f, vp, vp, C.POINTER(ErsdOpts), vp]
         L.ersd_verify_noalloc.argtypes = L.ersd_verify.argtypes
+        L.ersd_verify_tokens.argtypes = L.ersd_verify.argtypes
         L.ersd_verify_tree.argtypes = [vp, vp, i, C.POINTER(C.c_int32), vp, i, i, i, f, vp, vp,
                                        C.POINTER(ErsdOpts), vp]
         L.ersd_tree_depth.argtypes = [C.POINTER(C.c_int32), i]
@@ -74,7 +75,7 @@ def lib():
         L.ersd_workspace_init.argtypes = [vp, C.c_size_t, vp]
         L.ersd_status_string.argtypes = [i]
         L.ersd_status_string.restype = C.c_char_p
-        for name in ("ersd_race_sample", "ersd_verify", "ersd_verify_noalloc", "ersd_verify_tree", "ersd_tree_depth",
+        for name in ("ersd_race_sample", "ersd_verify", "ersd_verify_tokens", "ersd_verify_noalloc", "ersd_verify_tree", "ersd_tree_depth",
                      "ersd_row_keys", "ersd_workspace_init", "ersd_last_cuda_error", "ersd_version"):
             getattr(L, name).restype = i
         _lib = L
@@ -188,6 +189,24 @@ def ersd_verify(target_logits: torch.Tensor, draft_logits: Optional[torch.Tensor
                              _ptr(seeds), B, rows - 1, V, float(T), _ptr(out_tokens),
                              _ptr(out_accept_len), C.byref(opts) if opts is not None else None,
                              _stream(stream)), "ersd_verify")
+
+
+def ersd_verify_tokens(target_logits: torch.Tensor, draft_tokens: Optional[torch.Tensor], seeds: torch.Tensor,
+                       T: float, out_tokens: torch.Tensor, out_accept_len: torch.Tensor,
+                       opts: Optional[ErsdOpts] = None, stream=None) -> None:
+    """target [B, k+1, V], draft_tokens int32 [B, k] (drafted earlier with the same races),
+    out_tokens int32 [B, k+1], out_accept_len int32 [B]."""
+    _dev(target_logits, None, "target_logits")
+    B, rows, V = target_logits.shape
+    if draft_tokens is not None:
+        _dev(draft_tokens, torch.int32, "draft_tokens")
+    _dev(seeds, torch.int64, "seeds")
+    _dev(out_tokens, torch.int32, "out_tokens")
+    _dev(out_accept_len, torch.int32, "out_accept_len")
+    _check(lib().ersd_verify_tokens(_ptr(target_logits), _ptr(draft_tokens), _dtype_code(target_logits),
+                                    _ptr(seeds), B, rows - 1, V, float(T), _ptr(out_tokens),
+                                    _ptr(out_accept_len), C.byref(opts) if opts is not None else None,
+                                    _stream(stream)), "ersd_verify_tokens")
 
 
 def ersd_verify_noalloc(target_logits: torch.Tensor, draft_logits: Optional[torch.Tensor],

@@ -64,6 +64,7 @@ enum Mode { kSample = 0, kVerify = 1 };
 struct Params {
   const void* target;  // target logits (race_sample: the logits)
   const void* draft;
+  const int32_t* given_tok;  // [B, k] drafted tokens when they are given instead of draft rows
   int64_t ld_t, ld_d;
   const uint64_t* seeds;
   const uint32_t* seq_ids;
@@ -782,6 +783,12 @@ __device__ __noinline__ void finish_piece(const Params& p, const TreeDesc& tree)
       sh.dkey[m] = ok ? (float)L.key : INFINITY;
     }
   }
+  if (p.given_tok) {  // drafted earlier: node n holds the token drafted at position n - 1
+    for (int n = 1 + tid; n < p.rows; n += kThreads) {
+      sh.dtok[n] = p.given_tok[(size_t)b * (p.rows - 1) + (n - 1)];
+      sh.dkey[n] = INFINITY;
+    }
+  }
   if (tid == 0) {
     sh.dtok[0] = -1;
     sh.dkey[0] = INFINITY;
@@ -1107,13 +1114,14 @@ static void fill_common(Params& p, const ersd_opts& o, const uint64_t* seeds, in
 static int verify_impl(const void* target, const void* draft, int dt, const TreeDesc& tree, int D,
                        int cmax, bool chain, const uint64_t* seeds, int B, int rows, int draft_rows,
                        int V, float T, int32_t* out_tokens, int32_t* out_accept_len,
-                       const ersd_opts* opts, void* stream) {
+                       const ersd_opts* opts, void* stream, const int32_t* given_tok = nullptr) {
   const ersd_opts o = read_opts(opts);
   Params p;
   memset(&p, 0, sizeof p);
   fill_common(p, o, seeds, B, rows, V, T);
   p.target = target;
   p.draft = draft;
+  p.given_tok = given_tok;
   p.ld_t = o.ld_target ? o.ld_target : V;
   p.ld_d = o.ld_draft ? o.ld_draft : V;
   if (p.ld_t < V || p.ld_d < V) return ERSD_EINVAL;
@@ -1226,6 +1234,33 @@ int ersd_verify(const void* target_logits, const void* draft_logits, ersd_dtype 
   if (st != ERSD_OK) return st;
   return verify_impl(target_logits, draft_logits, dt, tree, D, cmax, true, seeds, B, k + 1, k, V, T,
                      out_tokens, out_accept_len, opts, cuda_stream);
+}
+
+int ersd_verify_tokens(const void* target_logits, const int32_t* draft_tokens, ersd_dtype dt,
+                       const uint64_t* seeds, int B, int k, int V, float T, int32_t* out_tokens,
+                       int32_t* out_accept_len, const ersd_opts* opts, void* cuda_stream) {
+  if (k < 0) return ERSD_EINVAL;
+  if (k + 1 > ERSD_MAX_ROWS) return ERSD_EUNSUPPORTED;
+  int st = check_common(target_logits, dt, seeds, B, k + 1, V, T);
+  if (st != ERSD_OK) return st;
+  if (!out_tokens || !out_accept_len) return ERSD_EINVAL;
+  if (k > 0) {
+    if (!draft_tokens) return ERSD_EINVAL;
+    if (((uintptr_t)draft_tokens & 3) != 0) return ERSD_EALIGN;
+  }
+  int32_t parent[ERSD_MAX_ROWS];
+  for (int n = 0; n <= k; ++n) parent[n] = n - 1;
+  TreeDesc tree;
+  int D = 0, cmax = 1;
+  st = build_tree(parent, k, &tree, &D, &cmax);
+  if (st != ERSD_OK) return st;
+  // the chain keeps its shape for the walk, but no row has a draft row to race
+  for (int n = 0; n <= k; ++n) {
+    tree.nchild[n] = 0;
+    tree.order[n] = (uint8_t)n;
+  }
+  return verify_impl(target_logits, nullptr, dt, tree, D, 1, true, seeds, B, k + 1, k, V, T, out_tokens,
+                     out_accept_len, opts, cuda_stream, k > 0 ? draft_tokens : nullptr);
 }
 
 int ersd_verify_tree(const void* target_logits, const void* draft_logits, ersd_dtype dt,

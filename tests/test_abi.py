@@ -108,6 +108,8 @@ def test_argument_errors_are_found_on_the_host(L):
     o.struct_size = C.sizeof(ErsdOpts)
     o.ld_target = 4                                                          # stride below V
     assert v(p, p, 1, p, 1, 2, 8, 1.0, p, p, C.byref(o), None) == EINVAL
+    assert L.ersd_verify_tokens(p, None, 1, p, 1, 2, 8, 1.0, p, p, None, None) == EINVAL      # k > 0 needs tokens
+    assert L.ersd_verify_tokens(p, C.c_void_p(4098), 1, p, 1, 2, 8, 1.0, p, p, None, None) == -2  # misaligned int32
     assert L.ersd_row_keys(None, 1, 8, 1.0, 0, 0, 0, 0, p, None) == EINVAL
     assert L.ersd_row_keys(p, 1, 8, 1.0, 0, 0, 0, 3, p, None) == EINVAL     # modes are 0, 1, 2
     assert L.ersd_workspace_init(None, 16, None) == EINVAL

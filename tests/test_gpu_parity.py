@@ -310,6 +310,62 @@ def test_race_sample_draft_then_verify_is_consistent(ersd):
     assert (tok[..., 0] == out["draft_tok"]).all()
 
 
+# ------------------------------------------------------------------ token-given verification
+@pytest.mark.parametrize("name,scale", [("c2", dict(B=6)), ("c5", dict(B=4)), ("c1", {})])
+def test_verify_tokens_against_the_oracle(ersd, name, scale):
+    """Draft with ersd_race_sample on the draft rows, then verify the tokens against the target
+    rows only; the oracle does the same two steps."""
+    import oracle
+    w = wl.scaled(wl.CONFIGS[name], **scale)
+    inp = to_dev(wl.make_inputs(w, call=91))
+    temps = inp.get("temps")
+    kw_d = {} if temps is None else dict(temps=temps[:, :w.k].contiguous(),
+                                          temp_strides=(w.k, 1))
+    drafted = torch.empty(w.B, w.k, 1, dtype=torch.int32, device="cuda")
+    ersd.ersd_race_sample(inp["draft"], inp["seeds"], inp["T"], drafted, ersd.make_opts(**kw_d))
+    dtok = drafted[..., 0].contiguous()
+    # spoil some drafted tokens so that rejections at every position occur
+    spoil = torch.zeros_like(dtok, dtype=torch.bool)
+    spoil[::3, 1] = True
+    dtok = torch.where(spoil, (dtok + 1) % w.V, dtok)
+    tok = torch.full((w.B, w.k + 1), -7, dtype=torch.int32, device="cuda")
+    acc = torch.full((w.B,), -7, dtype=torch.int32, device="cuda")
+    ttok = torch.empty(w.B, w.k + 1, dtype=torch.int32, device="cuda")
+    tkey = torch.empty(w.B, w.k + 1, dtype=torch.float32, device="cuda")
+    kw_t = {} if temps is None else dict(temps=temps, temp_strides=(temps.stride(0), temps.stride(1)))
+    for split in (0, 3):
+        ersd.ersd_verify_tokens(inp["target"], dtok, inp["seeds"], inp["T"], tok, acc,
+                                ersd.make_opts(out_target_tok=ttok, out_target_key=tkey, split_v=split, **kw_t))
+        torch.cuda.synchronize()
+        ref = oracle.verify_tokens(wl.as_numpy_logits(inp["target"]), dtok.cpu().numpy(),
+                                   wl.seeds_as_u64(inp["seeds"]), T=inp["T"],
+                                   temps=None if temps is None else temps.cpu().numpy())
+        gap = ref["target_key"][..., 1] - ref["target_key"][..., 0]
+        assert (gap >= 1e-5).all()                     # no near-tie in these inputs: exact comparison
+        assert (ttok.cpu().numpy() == ref["target_tok"]).all()
+        assert (tok.cpu().numpy() == ref["tokens"]).all()
+        assert (acc.cpu().numpy() == ref["accept_len"]).all()
+        assert np.abs(tkey.cpu().numpy() - ref["target_key"][..., 0]).max() <= KEY_TOL
+    # and it agrees with the row-given entry point when the tokens are the draft rows' winners
+    ersd.ersd_verify_tokens(inp["target"], drafted[..., 0].contiguous(), inp["seeds"], inp["T"], tok, acc,
+                            ersd.make_opts(**kw_t))
+    full = ersd.verify(inp["target"], inp["draft"], inp["seeds"], inp["T"], temps=temps)
+    torch.cuda.synchronize()
+    assert (tok == full["tokens"]).all() and (acc == full["accept_len"]).all()
+
+
+def test_verify_tokens_without_drafts(ersd):
+    w = wl.Workload("k0t", B=2, k=0, V=999, dtype="bf16", T=1.0, config_id=49)
+    inp = to_dev(wl.make_inputs(w))
+    tok = torch.empty(2, 1, dtype=torch.int32, device="cuda")
+    acc = torch.empty(2, dtype=torch.int32, device="cuda")
+    ersd.ersd_verify_tokens(inp["target"], None, inp["seeds"], 1.0, tok, acc, None)
+    ref = torch.empty(2, 1, 1, dtype=torch.int32, device="cuda")
+    ersd.ersd_race_sample(inp["target"], inp["seeds"], 1.0, ref, None)
+    torch.cuda.synchronize()
+    assert (tok[:, 0] == ref[:, 0, 0]).all() and (acc == 0).all()
+
+
 # ------------------------------------------------------------------ keys, workspace, repeats
 def test_row_keys_match_the_oracle(ersd):
     import oracle
