@@ -102,10 +102,13 @@ class ClockSampler:
                 "samples": len(inside)}
 
 
-def algorithmic_bytes(w, inp):
-    """Bytes one verify launch must read: every target row, every draft row that has children."""
+def algorithmic_bytes(w, inp, entry="verify"):
+    """Bytes one verify launch must read: every target row, every draft row that has children
+    (token-given verification reads target rows only)."""
     es = inp["target"].element_size()
-    if w.is_tree:
+    if entry == "tokens":
+        rows = w.B * w.rows_target
+    elif w.is_tree:
         parent = inp["parent"]
         internal = len({p for p in parent if p >= 0})
         rows = w.B * (w.rows_target + internal)
@@ -176,6 +179,9 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="c5")
+    ap.add_argument("--entry", default="verify", choices=["verify", "tokens"],
+                    help="verify: ersd_verify / ersd_verify_tree (the headline path); tokens: "
+                         "ersd_verify_tokens on tokens drafted before the timed region")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sets", type=int, default=3, help="distinct input sets rotated between launches")
     ap.add_argument("--e2e-steps", type=int, default=4)
@@ -228,9 +234,28 @@ def main():
 
     all_opts = [opts_for(inp) for inp in sets]
 
+    drafted = None
+    if args.entry == "tokens":
+        if w.is_tree:
+            raise SystemExit("--entry tokens takes a sequence workload")
+        drafted = []
+        for inp, o in zip(sets, all_opts):     # drafting happens before the timed region
+            d = torch.empty(w.B, w.k, 1, dtype=torch.int32, device="cuda")
+            kw = {}
+            if inp.get("temps") is not None:
+                t_d = inp["temps"][:, :w.k].contiguous()
+                kw = dict(temps=t_d, temp_strides=(t_d.stride(0), t_d.stride(1)))
+                inp["temps_draft"] = t_d
+            binding.ersd_race_sample(inp["draft"], inp["seeds"], inp["T"], d, binding.make_opts(**kw), stream)
+            drafted.append(d[..., 0].contiguous())
+        torch.cuda.synchronize()
+
     def step(i):
         inp = sets[i % len(sets)]
-        if w.is_tree:
+        if drafted is not None:
+            binding.ersd_verify_tokens(inp["target"], drafted[i % len(sets)], inp["seeds"], inp["T"], tokens,
+                                       accept, all_opts[i % len(sets)], stream)
+        elif w.is_tree:
             binding.ersd_verify_tree(inp["target"], inp["draft"], inp["parent"], inp["seeds"], inp["T"],
                                      tokens, accept, all_opts[i % len(sets)], stream)
         else:
@@ -267,27 +292,34 @@ def main():
 
     # ---- roofline of the one kernel a step launches
     peak, peak_kind = load_peaks()
-    alg_bytes = algorithmic_bytes(w, sets[0])
+    alg_bytes = algorithmic_bytes(w, sets[0], args.entry)
     achieved = alg_bytes / (ms_step * 1e-3) / 1e9
     # DRAM traffic per launch from the ncu capture summarised in profiles/ (dram read + write bytes
     # over algorithmic bytes, taken on this workload); void once the kernel has changed since
     traffic = None
-    if binding.ersd_version() == TRAFFIC_AT_VERSION:
+    if binding.ersd_version() == TRAFFIC_AT_VERSION and args.entry == "verify" and args.workload == "c5":
         traffic = DRAM_BYTES_PER_ALGORITHMIC_BYTE * alg_bytes
     # the other roof: every vocabulary index needs a quarter of a Philox4x32-10 call, 4.5 wide
     # multiplies and 4.75 three-input xors on the integer path (64 lanes per clock and SM)
     n_index = w.B * w.rows_target * w.V
     t_alu_ms = n_index * 9.25 / (64.0 * SM_COUNT * (clocks["sm_max_mhz"] or 1965.0) * 1e6) * 1e3
+    t_hbm_ms = alg_bytes / (peak * 1e9) * 1e3
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": traffic, "peak_kind": peak_kind + " copy bandwidth",
                 "algorithmic_bytes_per_launch": alg_bytes, "kernel": "ersd_race_kernel<bf16>",
-                "kernel_ms": ms_step, "t_hbm_ms": alg_bytes / (peak * 1e9) * 1e3,
-                "t_int_ms": t_alu_ms,
+                "kernel_ms": ms_step, "t_hbm_ms": t_hbm_ms, "t_int_ms": t_alu_ms,
                 "note": "t_int_ms: Philox integer work alone at the nominal 64 int lanes/clk/SM"}
+    if t_alu_ms > t_hbm_ms:
+        # fewer bytes per index than integer work (target rows only): the integer path is the roof
+        int_ops = n_index * 9.25
+        peak_ops = 64.0 * SM_COUNT * (clocks["sm_max_mhz"] or 1965.0) * 1e6 / 1e9
+        roofline.update(bound="alu", achieved=int_ops / (ms_step * 1e-3) / 1e9, peak=peak_ops, unit="Gop/s",
+                        frac=t_alu_ms / ms_step, traffic=None,
+                        peak_kind="64 integer lanes per clock and SM x 148 SMs x max SM clock")
 
     # ---- end to end: host buffers in pinned memory, copies inside the timed region
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and args.entry == "verify":
         h = sets[0]
         host_t = h["target"].cpu().pin_memory()
         host_d = h["draft"].cpu().pin_memory()
@@ -329,7 +361,9 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32 screen + f64 decision, u32 Philox", "data": "synthetic",
-            "config": workload_config(w, "inputs larger than L2; %d input sets rotated" % len(sets)),
+            "config": dict(workload_config(w, "inputs larger than L2; %d input sets rotated" % len(sets)),
+                           entry="ersd_verify_tokens" if args.entry == "tokens" else
+                           ("ersd_verify_tree" if w.is_tree else "ersd_verify")),
             "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps, "roofline": roofline,
             "cpu_baseline": cpu, "mean_accept_len": mean_accept}))
     if dist is not None:
