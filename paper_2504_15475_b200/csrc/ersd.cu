@@ -595,15 +595,47 @@ __device__ __forceinline__ void stream_piece(const char* const* rows, bool ring_
   }
 }
 
-// Merge `n` sorted partial lists of `c` entries each (global memory written by other blocks)
-// into a fresh warp list.
+// Merge `n` sorted partial lists of `c` entries each (global memory written by other blocks,
+// n * c <= 64) into a fresh warp list.  All entries are fetched at once, two per lane, so the
+// merge pays one memory round trip, not one per entry.
 __device__ __forceinline__ void merge_partials(WarpList& L, const Entry* part, int n, int c,
                                                int lane) {
+  const int total = n * c;
+  double k0 = (double)INFINITY, k1 = (double)INFINITY;
+  int i0 = 0x7FFFFFFF, i1 = 0x7FFFFFFF;  // unused slots carry idx = INT_MAX
+  if (lane < total) {
+    k0 = __ldcg(&part[lane].key);
+    i0 = __ldcg(&part[lane].idx);
+  }
+  if (lane + 32 < total) {
+    k1 = __ldcg(&part[lane + 32].key);
+    i1 = __ldcg(&part[lane + 32].idx);
+  }
   L.init();
-  for (int e = 0; e < n * c; ++e) {
-    const double k = __ldcg(&part[e].key);
-    const int i = __ldcg(&part[e].idx);
-    if (i != 0x7FFFFFFF) L.insert(k, i, lane);  // unused slots carry idx = INT_MAX
+  if (c == 1) {  // winners only: the smallest (key, idx) by a shuffle tree, result in lane 0
+    if (k1 < k0 || (k1 == k0 && i1 < i0)) {
+      k0 = k1;
+      i0 = i1;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      const double ok = __shfl_down_sync(kFull, k0, off);
+      const int oi = __shfl_down_sync(kFull, i0, off);
+      if (ok < k0 || (ok == k0 && oi < i0)) {
+        k0 = ok;
+        i0 = oi;
+      }
+    }
+    if (lane == 0) {
+      L.key = k0;
+      L.idx = i0;
+    }
+    return;
+  }
+  for (int e = 0; e < total; ++e) {
+    const double k = __shfl_sync(kFull, e < 32 ? k0 : k1, e & 31);
+    const int i = __shfl_sync(kFull, e < 32 ? i0 : i1, e & 31);
+    if (i != 0x7FFFFFFF) L.insert(k, i, lane);
   }
 }
 
