@@ -558,15 +558,14 @@ __device__ __noinline__ void first_tile(int stage, int i0, int vend, float c2, f
   unsigned bits = 0;
 #pragma unroll
   for (int r = 0; r < NR; ++r)
-    if (!(fmaf(-zub[r], c2, lgm) > *(volatile float*)&sh.lim[r])) bits |= 1u << r;
+    if (fmaf(-zub[r], c2, lgm) <= *(volatile float*)&sh.lim[r]) bits |= 1u << r;
   if (__any_sync(kFull, bits != 0)) settle_tile<DT>(stage, i0, bits, c2, T);
 }
 
 // One piece = chunk [v0, v1) of a logit row (NR = 1) or of a draft/target pair (NR = 2); rows[]
-// point at the rows' first elements.  The streaming loop takes the full tiles after the first
-// (its trip count depends only on launch parameters, which keeps the loop control on the
-// uniform datapath); the first tile yields the first threshold unless an earlier chunk of the
-// row handed one down; a ragged last tile is looked at index by index.
+// point at the rows' first elements.  The streaming loop takes the full tiles after the first;
+// the first tile yields the first threshold unless an earlier chunk of the row handed one down;
+// a ragged last tile gets the cheap test with bounds-checked loads.
 // (Inlined into the kernel, whose other parts are out-of-line calls: the loop then gets a
 // register allocation of its own.)
 template <int DT, int NR>
@@ -589,7 +588,15 @@ __device__ __forceinline__ void stream_piece(const char* const* rows, bool ring_
     else edge_tile<DT, NR>(kStages - 1, i0, v1, c2, T);
     if (nfull > 1) st.run(i0 + kTile, c2, T);
     cp_async_wait<0>();
-    if (ntiles > nfull && ntiles > 1) edge_tile<DT, NR>(0, i0 + (ntiles - 1) * kTile, v1, c2, T);
+    if (ntiles > nfull && ntiles > 1) {
+      // ragged last tile: the cheap test again (indices beyond the row read as NaN and never
+      // pass) unless the chunk still has no threshold
+      bool tau_now = true;
+#pragma unroll
+      for (int r = 0; r < NR; ++r) tau_now = tau_now && (*(volatile float*)&sh->tau[r] < INFINITY);
+      if (tau_now) first_tile<DT, NR>(0, i0 + (ntiles - 1) * kTile, v1, c2, T);
+      else edge_tile<DT, NR>(0, i0 + (ntiles - 1) * kTile, v1, c2, T);
+    }
   } else {
     for (int t = 0; t < ntiles; ++t, i0 += kTile) edge_tile<DT, NR>(0, i0, v1, c2, T);
   }
