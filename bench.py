@@ -125,16 +125,39 @@ def oracle_rate(w, inp, n_seq, reps=1):
     drf = wl.as_numpy_logits(inp["draft"][:n_seq])
     seeds = wl.seeds_as_u64(inp["seeds"][:n_seq])
     temps = None if inp.get("temps") is None else inp["temps"][:n_seq].cpu().numpy()
-    best = None
+    best, ref = None, None
     for _ in range(reps):
         t0 = time.perf_counter()
         if w.is_tree:
-            oracle.verify_tree(tgt, drf, inp["parent"], seeds, T=inp["T"], temps=temps)
+            ref = oracle.verify_tree(tgt, drf, inp["parent"], seeds, T=inp["T"], temps=temps)
         else:
-            oracle.verify(tgt, drf, seeds, T=inp["T"], temps=temps)
+            ref = oracle.verify(tgt, drf, seeds, T=inp["T"], temps=temps)
         dt = time.perf_counter() - t0
         best = dt if best is None else min(best, dt)
-    return n_seq * w.rows_target / best, best, oracle.max_threads()
+    return n_seq * w.rows_target / best, best, oracle.max_threads(), ref
+
+
+def parity_report(w, inp, n_seq, ref):
+    """The library's result on the oracle's sample against the oracle's: target winners of every
+    row, accepted lengths and emitted tokens.  A row counts as a near-tie when the oracle's two
+    best keys are closer than 1e-5 (either winner is right there)."""
+    import numpy as np
+    from paper_2504_15475_b200 import binding
+    out = binding.verify(inp["target"][:n_seq], inp["draft"][:n_seq], inp["seeds"][:n_seq], inp["T"],
+                         temps=None if inp.get("temps") is None else inp["temps"][:n_seq].contiguous(),
+                         parent=inp.get("parent"), want_rows=True)
+    ttok = out["target_tok"].cpu().numpy()
+    gap = ref["target_key"][..., 1] - ref["target_key"][..., 0]
+    differ = ttok != ref["target_tok"]
+    acc_same = out["accept_len"].cpu().numpy() == ref["accept_len"]
+    tok_same = (out["tokens"].cpu().numpy() == ref["tokens"]).all(axis=1)
+    key_err = float(np.abs(out["target_key"].cpu().numpy()[~differ] - ref["target_key"][..., 0][~differ]).max())
+    return {"sequences_checked": int(n_seq), "target_rows_checked": int(ttok.size),
+            "oracle_near_tie_rows": int((gap < 1e-5).sum()),
+            "winner_mismatches": int(differ.sum()),
+            "winner_mismatches_outside_near_ties": int((differ & ~(gap < 1e-5)).sum()),
+            "sequences_with_other_accept_len_or_tokens": int((~(acc_same & tok_same)).sum()),
+            "max_winner_key_error": key_err}
 
 
 def run_reference(args, w):
@@ -343,11 +366,12 @@ def main():
                "steps": args.e2e_steps}
 
     # ---- the oracle on the host cores, on a bounded sample of the same workload (rank 0, N = 1)
-    cpu = None
+    cpu, parity = None, None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         n_seq = w.B if args.cpu_seqs <= 0 else max(1, min(w.B, args.cpu_seqs))
         t_cpu0 = time.perf_counter()
         rates = [oracle_rate(w, sets[0], n_seq) for _ in range(max(1, args.cpu_passes))]
+        parity = parity_report(w, sets[0], n_seq, rates[-1][3]) if args.entry == "verify" else None
         t_cpu = time.perf_counter() - t_cpu0
         rate = statistics.median(r[0] for r in rates)
         cores = rates[0][2]
@@ -365,7 +389,7 @@ def main():
                            entry="ersd_verify_tokens" if args.entry == "tokens" else
                            ("ersd_verify_tree" if w.is_tree else "ersd_verify")),
             "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps, "roofline": roofline,
-            "cpu_baseline": cpu, "mean_accept_len": mean_accept}))
+            "cpu_baseline": cpu, "parity_on_cpu_sample": parity, "mean_accept_len": mean_accept}))
     if dist is not None:
         dist.destroy_process_group()
 
