@@ -574,8 +574,8 @@ __device__ __forceinline__ void stream_piece(const char* const* rows, bool ring_
   constexpr int kStages = Geo<DT>::kStages;
   Shared<DT>* sh = &block_state<DT>();
   const int tid = threadIdx.x;
-  const int ntiles = (v1 - v0 + kTile - 1) / kTile;
-  const int nfull = (v1 - v0) / kTile;       // tiles that lie fully inside the piece
+  const int ntiles = (int)((unsigned)(v1 - v0 + kTile - 1) / kTile);
+  const int nfull = (int)((unsigned)(v1 - v0) / kTile);  // tiles that lie fully inside the piece
   int i0 = v0 + tid * kPerThread;
   if (ring_ok) {
     Streamer<DT, NR> st;
@@ -656,11 +656,7 @@ __device__ __noinline__ void setup_piece(const Params& p, const TreeDesc& tree) 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // every thread decodes (cheap, no memory); single lanes of different warps then fill in the
   // parts of the state side by side, so that their memory latencies overlap
-  const int n_units = p.B * p.rows;
-  const int s = blockIdx.x / n_units;
-  const int rem = blockIdx.x - s * n_units;
-  const int ri = rem / p.B;
-  const int b = rem - ri * p.B;
+  const int s = blockIdx.z, ri = blockIdx.y, b = blockIdx.x;  // (no division: keeps these uniform)
   const int r = (p.mode == kSample) ? ri : (int)tree.order[ri];
   const int unit = b * p.rows + r;
   const int cq = (p.mode == kSample) ? 0 : (int)tree.nchild[r];
@@ -885,11 +881,7 @@ __global__ void __launch_bounds__(kThreads, ERSD_MIN_BLOCKS)
 ersd_race_kernel(const __grid_constant__ Params p, const __grid_constant__ TreeDesc tree) {
   // The same decode as in setup_piece, from launch parameters only: everything here is uniform
   // over the block, and the compiler can tell.
-  const int n_units = p.B * p.rows;
-  const int s = blockIdx.x / n_units;
-  const int rem = blockIdx.x - s * n_units;
-  const int ri = rem / p.B;
-  const int b = rem - ri * p.B;
+  const int s = blockIdx.z, ri = blockIdx.y, b = blockIdx.x;  // (no division: keeps these uniform)
   const int r = (p.mode == kSample) ? ri : (int)tree.order[ri];
   const int cq = (p.mode == kSample) ? 0 : (int)tree.nchild[r];
   const int v0 = s * p.per_chunk;
@@ -1113,12 +1105,14 @@ static int prefer_shared_memory() {
 }
 
 static int launch(const Params& p, const TreeDesc& tree, int dt, cudaStream_t st) {
-  const int64_t items = (int64_t)p.B * p.rows * p.S;
-  if (items > 0x7FFFFFFF) return ERSD_EINVAL;
+  // grid (sequence, row in launch order, chunk): blocks are dispatched x fastest, z slowest, which
+  // is the chunk-major order the kernel counts on, and the kernel needs no division to decode
+  if (p.rows > 65535 || p.S > 65535) return ERSD_EUNSUPPORTED;
+  const dim3 grid((unsigned)p.B, (unsigned)p.rows, (unsigned)p.S);
   const int pst = prefer_shared_memory();
   if (pst != ERSD_OK) return pst;
-  if (dt == ERSD_BF16) ersd_race_kernel<ERSD_BF16><<<(unsigned)items, kThreads, sizeof(Shared<ERSD_BF16>), st>>>(p, tree);
-  else ersd_race_kernel<ERSD_F32><<<(unsigned)items, kThreads, sizeof(Shared<ERSD_F32>), st>>>(p, tree);
+  if (dt == ERSD_BF16) ersd_race_kernel<ERSD_BF16><<<grid, kThreads, sizeof(Shared<ERSD_BF16>), st>>>(p, tree);
+  else ersd_race_kernel<ERSD_F32><<<grid, kThreads, sizeof(Shared<ERSD_F32>), st>>>(p, tree);
   const cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? ERSD_OK : cuda_fail(e);
 }
