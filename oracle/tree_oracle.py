@@ -1,0 +1,89 @@
+"""Oracle for the optimal draft tree (TEST INFRASTRUCTURE, not product code).
+
+Section 4 ("Markov Chain Simulation") defines the optimal tree with k + 1 vertices as the one that
+maximises the sum of its vertices' acceptance probabilities R(j); because a vertex can only be
+accepted when its ancestors are, R never grows along a path, and the optimum is the set of the k
+vertices of highest R.  This file writes that definition out -- enumerate, sort, take k -- for
+the 0-th order model the paper's experiments use, R(j_1..j_m) = a[j_1] * ... * a[j_m] with a[r]
+the acceptance probability of a node's child of rank r.  It does not follow Algorithm 3's
+priority queue (the library does); `best_tree_by_search` is an exhaustive search over all trees
+for tiny k that pins the definition itself.
+"""
+from __future__ import annotations
+
+import itertools
+from typing import Dict, List, Sequence, Tuple
+
+
+def vertex_probability(path: Tuple[int, ...], accept: Sequence[float]) -> float:
+    r = 1.0
+    for j in path:
+        r *= accept[j] if j < len(accept) else 0.0
+    return r
+
+
+def top_k_vertices(accept: Sequence[float], k: int) -> List[Tuple[float, Tuple[int, ...]]]:
+    """The k vertices of highest R (ties: shallower first, then lexicographic), each (R, path)."""
+    C = len(accept)
+    cand = []
+    for depth in range(1, k + 1):
+        # a vertex of rank r at some level needs r + depth <= k vertices before it can be in a
+        # k-vertex prefix-closed set, which bounds the enumeration
+        for path in itertools.product(range(min(C, k)), repeat=depth):
+            if sum(j + 1 for j in path) <= k:
+                cand.append((vertex_probability(path, accept), path))
+    cand.sort(key=lambda t: (-t[0], len(t[1]), t[1]))
+    return cand[:k]
+
+
+def expected_accepted(paths, accept: Sequence[float]) -> float:
+    return sum(vertex_probability(tuple(p), accept) for p in paths)
+
+
+def is_valid_tree(paths) -> bool:
+    """Prefix-closed and sibling-closed: a vertex needs its parent and its previous sibling."""
+    s = {tuple(p) for p in paths}
+    for p in s:
+        if len(p) > 1 and p[:-1] not in s:
+            return False
+        if p[-1] > 0 and p[:-1] + (p[-1] - 1,) not in s:
+            return False
+    return True
+
+
+def best_tree_by_search(accept: Sequence[float], k: int) -> float:
+    """Largest expected number of accepted tokens over ALL valid trees with k drafted vertices."""
+    C = len(accept)
+    best = 0.0
+
+    seen: Dict[frozenset, bool] = {}
+
+    def grow_memo(tree: frozenset, total: float):
+        if tree in seen:
+            return
+        seen[tree] = True
+        nonlocal best
+        if len(tree) == k:
+            best = max(best, total)
+            return
+        frontier = set()
+        for p in list(tree) + [()]:
+            child = p + (0,)
+            if child not in tree:
+                frontier.add(child)
+            if p:
+                sib = p[:-1] + (p[-1] + 1,)
+                if sib[-1] < C and sib not in tree:
+                    frontier.add(sib)
+        for v in frontier:
+            grow_memo(tree | {v}, total + vertex_probability(v, accept))
+
+    grow_memo(frozenset(), 0.0)
+    return best
+
+
+def parent_array(paths) -> List[int]:
+    """Vertices in lexicographic order (the paper's order) as a parent-index array, root first."""
+    order = [()] + sorted(tuple(p) for p in paths)
+    index = {p: n for n, p in enumerate(order)}
+    return [-1] + [index[p[:-1]] for p in order[1:]]
