@@ -11,7 +11,6 @@ for tiny k that pins the definition itself.
 """
 from __future__ import annotations
 
-import itertools
 from typing import Dict, List, Sequence, Tuple
 
 
@@ -26,12 +25,18 @@ def top_k_vertices(accept: Sequence[float], k: int) -> List[Tuple[float, Tuple[i
     """The k vertices of highest R (ties: shallower first, then lexicographic), each (R, path)."""
     C = len(accept)
     cand = []
-    for depth in range(1, k + 1):
-        # a vertex of rank r at some level needs r + depth <= k vertices before it can be in a
-        # k-vertex prefix-closed set, which bounds the enumeration
-        for path in itertools.product(range(min(C, k)), repeat=depth):
-            if sum(j + 1 for j in path) <= k:
-                cand.append((vertex_probability(path, accept), path))
+
+    def extend(path, need):
+        # `need` = vertices a valid tree must hold to contain `path` (it with its ancestors and
+        # all their earlier siblings); only vertices with need <= k can be in a k-vertex tree
+        for j in range(C):
+            if need + j + 1 > k:
+                break
+            child = path + (j,)
+            cand.append((vertex_probability(child, accept), child))
+            extend(child, need + j + 1)
+
+    extend((), 0)
     cand.sort(key=lambda t: (-t[0], len(t[1]), t[1]))
     return cand[:k]
 
