@@ -216,6 +216,28 @@ int ersd_verify_noalloc(const void* target_logits, const void* draft_logits, ers
                         const uint64_t* seeds, int B, int k, int V, float T, int32_t* out_tokens,
                         int32_t* out_accept_len, const ersd_opts* opts, void* cuda_stream);
 
+/*
+ * Draft tree with the largest expected number of accepted tokens (Algorithm 3,
+ * "Optimal tree construction", Section 4).  HOST function, no GPU work.
+ * Acceptance probabilities follow the 0-th order model of the paper's
+ * experiments: a vertex reached through child ranks (j_1, .., j_m) is accepted
+ * with probability accept[j_1] * ... * accept[j_m], where accept[r] (HOST array
+ * of max_children doubles in [0, 1], non-increasing in r) is the probability
+ * that a verified node's child of rank r -- the (r+1)-th arrival of its race
+ * under the draft row -- is accepted.  Vertices are added greedily by
+ * probability from a priority queue; a chosen vertex offers its first child and
+ * its next sibling (ties: shallower first, then lexicographic).
+ *   parent_out  HOST [k + 1]: parent_out[0] = -1, vertices in lexicographic
+ *               order, so parent_out[n] < n and siblings ascend by rank -- the
+ *               form ersd_verify_tree takes.
+ *   expected_tokens  HOST, nullable: sum of the k vertices' probabilities.
+ * Errors: ERSD_EINVAL (null pointers, k < 0, max_children < 1, accept outside
+ * [0, 1] or increasing); ERSD_EUNSUPPORTED for k + 1 > ERSD_MAX_ROWS.  Ranks
+ * beyond ERSD_MAX_TOP_C are ignored.
+ */
+int ersd_optimal_tree(const double* accept, int max_children, int k, int32_t* parent_out,
+                      double* expected_tokens);
+
 /* Depth (longest root-to-leaf edge count) of a HOST parent array, or -1 if it is malformed. */
 int ersd_tree_depth(const int32_t* parent, int N);
 

@@ -22,7 +22,7 @@ ERSD_MAX_TOP_C, ERSD_MAX_ROWS, ERSD_MAX_SPLIT = 32, 256, 32
 ERSD_NOALLOC_MAX_ROWS = 1024
 ERSD_ENOALLOC_LIMIT = -6
 
-EXPORTS = ("ersd_race_sample", "ersd_verify", "ersd_verify_tokens", "ersd_verify_noalloc", "ersd_verify_tree", "ersd_tree_depth",
+EXPORTS = ("ersd_race_sample", "ersd_verify", "ersd_verify_tokens", "ersd_verify_noalloc", "ersd_verify_tree", "ersd_tree_depth", "ersd_optimal_tree",
            "ersd_row_keys", "ersd_workspace_bytes", "ersd_workspace_init", "ersd_status_string",
            "ersd_last_cuda_error", "ersd_version")
 
@@ -69,6 +69,8 @@ def lib():
         L.ersd_verify_tree.argtypes = [vp, vp, i, C.POINTER(C.c_int32), vp, i, i, i, f, vp, vp,
                                        C.POINTER(ErsdOpts), vp]
         L.ersd_tree_depth.argtypes = [C.POINTER(C.c_int32), i]
+        L.ersd_optimal_tree.argtypes = [C.POINTER(C.c_double), i, i, C.POINTER(C.c_int32), C.POINTER(C.c_double)]
+        L.ersd_optimal_tree.restype = i
         L.ersd_row_keys.argtypes = [vp, i, i, f, C.c_uint64, C.c_uint32, C.c_uint32, i, vp, vp]
         L.ersd_workspace_bytes.argtypes = [i, i]
         L.ersd_workspace_bytes.restype = C.c_size_t
@@ -160,6 +162,16 @@ def ersd_workspace_init(workspace: torch.Tensor, stream=None) -> None:
 def ersd_tree_depth(parent: Sequence[int]) -> int:
     arr = (C.c_int32 * len(parent))(*[int(p) for p in parent])
     return int(lib().ersd_tree_depth(arr, len(parent) - 1))
+
+
+def ersd_optimal_tree(accept: Sequence[float], k: int):
+    """(parent array [k + 1], expected number of accepted tokens) of the best k-token draft tree for
+    per-rank acceptance probabilities `accept` (host function, Algorithm 3)."""
+    a = (C.c_double * len(accept))(*[float(x) for x in accept])
+    parent = (C.c_int32 * (k + 1))()
+    expected = C.c_double(0.0)
+    _check(lib().ersd_optimal_tree(a, len(accept), int(k), parent, C.byref(expected)), "ersd_optimal_tree")
+    return list(parent), float(expected.value)
 
 
 def ersd_race_sample(logits: torch.Tensor, seeds: torch.Tensor, T: float, out_tok: torch.Tensor,
