@@ -274,6 +274,17 @@ def test_tree_shapes(ersd, parent):
     check_verify(inp, out)
 
 
+def test_tree_built_by_the_library_runs_through_tree_verification(ersd):
+    """Algorithm 3's tree for a measured-looking acceptance profile, verified with Algorithm 5."""
+    parent, expected = ersd.ersd_optimal_tree([0.55, 0.2, 0.1, 0.05], 14)
+    assert expected > 1.0
+    w = wl.Workload("opt_tree", B=4, k=14, V=12000, dtype="bf16", sigma=0.8, T=1.0, config_id=50,
+                    parent=tuple(parent))
+    inp = wl.make_inputs(w)
+    out = run_verify(ersd, inp)
+    check_verify(inp, out)
+
+
 def test_wide_star_uses_many_arrivals(ersd):
     parent = wl.star_parent(32)
     w = wl.Workload("star32", B=3, k=32, V=5000, dtype="f32", sigma=0.5, T=1.0, config_id=47,
