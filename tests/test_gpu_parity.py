@@ -208,6 +208,31 @@ def test_row_strides_and_unaligned_rows(ersd):
         assert (tok.cpu().numpy() == ref["tokens"]).all()
 
 
+def test_padded_rows_on_the_vector_path_and_many_small_sequences(ersd):
+    import oracle
+    # row stride larger than V but 16-byte aligned: the cp.async ring with a stride
+    B, k, V, ld = 3, 4, 6000, 6016
+    g = torch.Generator().manual_seed(21)
+    big_t = (torch.randn(B, k + 1, ld, generator=g) * 2).to(torch.bfloat16)
+    big_d = (torch.randn(B, k, ld, generator=g) * 2).to(torch.bfloat16)
+    seeds = wl.make_seeds(9, 1, B)
+    tok = torch.empty(B, k + 1, dtype=torch.int32, device="cuda")
+    acc = torch.empty(B, dtype=torch.int32, device="cuda")
+    for split in (0, 2):
+        ersd.ersd_verify(big_t.cuda(), big_d.cuda(), seeds.cuda(), 0.8, tok, acc,
+                         ersd.make_opts(ld_target=ld, ld_draft=ld, split_v=split))
+        torch.cuda.synchronize()
+        ref = oracle.verify(wl.as_numpy_logits(big_t[:, :, :V].contiguous()),
+                            wl.as_numpy_logits(big_d[:, :, :V].contiguous()), wl.seeds_as_u64(seeds), T=0.8)
+        assert (tok.cpu().numpy() == ref["tokens"]).all() and (acc.cpu().numpy() == ref["accept_len"]).all()
+    # many short sequences, long drafts: more work items than block slots, deep chain
+    w = wl.Workload("many", B=700, k=20, V=2500, dtype="bf16", sigma=0.4, T=1.0, config_id=51)
+    inp = wl.make_inputs(w)
+    out = run_verify(ersd, inp)
+    check_verify(inp, out)
+    assert out["accept_len"].max().item() >= 3
+
+
 def test_special_values(ersd):
     V = 300
     g = torch.Generator().manual_seed(9)
