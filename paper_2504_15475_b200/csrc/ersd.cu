@@ -25,7 +25,10 @@
 
 namespace ersd {
 
-constexpr int kThreads = 256;
+#ifndef ERSD_THREADS
+#define ERSD_THREADS 256
+#endif
+constexpr int kThreads = ERSD_THREADS;
 constexpr int kWarps = kThreads / 32;
 constexpr int kPerThread = 8;
 constexpr int kTile = kThreads * kPerThread;  // vocabulary indices per block iteration
@@ -687,13 +690,14 @@ __device__ __noinline__ void setup_piece(const Params& p, const TreeDesc& tree) 
                               : nullptr;
       sh.role[1].c = cq > 0 ? cq : 1;
       sh.role[1].aligned = p.aligned_d;
-    } else if (warp == 3 || warp == 4) {
-      // thresholds handed down by earlier chunks of this row (any of them is a valid bound)
-      const int q = warp - 3;
-      const float tau = (p.S > 1) ? tau_of_code(__ldcg(&p.slots[unit].tau_code[q])) : INFINITY;
-      sh.tau[q] = tau;
-      sh.lim[q] = (tau < INFINITY) ? lim_of_tau(tau) : INFINITY;
     }
+  }
+  if (warp == 3 && lane < 2) {
+    // thresholds handed down by earlier chunks of this row (any of them is a valid bound)
+    const int q = lane;
+    const float tau = (p.S > 1) ? tau_of_code(__ldcg(&p.slots[unit].tau_code[q])) : INFINITY;
+    sh.tau[q] = tau;
+    sh.lim[q] = (tau < INFINITY) ? lim_of_tau(tau) : INFINITY;
   }
   Entry e;
   e.key = (double)INFINITY;
@@ -723,7 +727,7 @@ __device__ __noinline__ void finish_piece(const Params& p, const TreeDesc& tree)
       L.key = lane < kWarps ? sh.list[role][lane][0].key : (double)INFINITY;
       L.idx = lane < kWarps ? sh.list[role][lane][0].idx : 0x7FFFFFFF;
 #pragma unroll
-      for (int off = kWarps / 2; off > 0; off >>= 1) {
+      for (int off = 16; off > 0; off >>= 1) {
         const double ok = __shfl_down_sync(kFull, L.key, off);
         const int oi = __shfl_down_sync(kFull, L.idx, off);
         if (ok < L.key || (ok == L.key && oi < L.idx)) {
