@@ -84,7 +84,7 @@ typedef struct ersd_opts {
   uint32_t struct_size;
   uint32_t top_c;          /* ersd_race_sample: arrivals per row, 0 or 1 = winner only */
   uint32_t split_v;        /* thread blocks per row; 0 = chosen by the library */
-  uint32_t reserved0;
+  uint32_t block_threads;  /* threads per block of the race kernel: 128, 256, or 0 = chosen by the library */
   int64_t ld_target;       /* row stride in elements of target_logits / logits; 0 = V */
   int64_t ld_draft;        /* row stride in elements of draft_logits; 0 = V */
   const float* temps;      /* device; temperature of row (b, r) = temps[b*temp_stride_b + r*temp_stride_r] */

@@ -30,7 +30,7 @@ EXPORTS = ("ersd_race_sample", "ersd_verify", "ersd_verify_tokens", "ersd_verify
 class ErsdOpts(C.Structure):
     _fields_ = [
         ("struct_size", C.c_uint32), ("top_c", C.c_uint32), ("split_v", C.c_uint32),
-        ("reserved0", C.c_uint32),
+        ("block_threads", C.c_uint32),
         ("ld_target", C.c_int64), ("ld_draft", C.c_int64),
         ("temps", C.c_void_p), ("temp_stride_b", C.c_int64), ("temp_stride_r", C.c_int64),
         ("seq_ids", C.c_void_p), ("pos_offsets", C.c_void_p),
@@ -116,14 +116,14 @@ def _dev(t: torch.Tensor, dtype, name: str):
     return t
 
 
-def make_opts(*, top_c: int = 0, split_v: int = 0, ld_target: int = 0, ld_draft: int = 0,
+def make_opts(*, top_c: int = 0, split_v: int = 0, block_threads: int = 0, ld_target: int = 0, ld_draft: int = 0,
               temps: Optional[torch.Tensor] = None, temp_strides: Sequence[int] = (0, 0),
               seq_ids: Optional[torch.Tensor] = None, pos_offsets: Optional[torch.Tensor] = None,
               out_draft_tok=None, out_draft_key=None, out_target_tok=None, out_target_key=None,
               out_path=None, out_key=None, workspace: Optional[torch.Tensor] = None) -> ErsdOpts:
     o = ErsdOpts()
     o.struct_size = C.sizeof(ErsdOpts)
-    o.top_c, o.split_v = top_c, split_v
+    o.top_c, o.split_v, o.block_threads = top_c, split_v, block_threads
     o.ld_target, o.ld_draft = ld_target, ld_draft
     if temps is not None:
         _dev(temps, torch.float32, "temps")
@@ -269,14 +269,14 @@ def ersd_row_keys(row: torch.Tensor, T: float, seed: int, seq_id: int, position:
 
 # --------------------------------------------------------------------------- conveniences
 def verify(target_logits, draft_logits, seeds, T=1.0, temps=None, parent=None, split_v=0,
-           want_rows=False, seq_ids=None, pos_offsets=None):
+           want_rows=False, seq_ids=None, pos_offsets=None, block_threads=0):
     """Allocate outputs, call ersd_verify / ersd_verify_tree, return a dict of device tensors."""
     B, rows, V = target_logits.shape
     dev = target_logits.device
     D = rows - 1 if parent is None else ersd_tree_depth(parent)
     out = dict(tokens=torch.empty(B, D + 1, dtype=torch.int32, device=dev),
                accept_len=torch.empty(B, dtype=torch.int32, device=dev))
-    kw = dict(split_v=split_v, seq_ids=seq_ids, pos_offsets=pos_offsets)
+    kw = dict(split_v=split_v, block_threads=block_threads, seq_ids=seq_ids, pos_offsets=pos_offsets)
     if temps is not None:
         kw.update(temps=temps, temp_strides=(temps.stride(0), temps.stride(1)))
     if want_rows:

@@ -159,20 +159,41 @@ def test_acceptance_tracks_the_closed_form_at_full_vocabulary(ersd):
 
 
 # ------------------------------------------------------------------ edge cases
-@pytest.mark.parametrize("V", [1, 2, 3, 5, 7, 8, 9, 31, 2047, 2048, 2049, 4100, 20000])
+@pytest.mark.parametrize("V", [1, 2, 3, 5, 7, 8, 9, 31, 1023, 1024, 1025, 2047, 2048, 2049, 4100, 20000])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_small_and_ragged_vocabularies(ersd, V, dtype):
     w = wl.Workload("edge", B=3, k=3, V=V, dtype=dtype, sigma=0.7, T=0.9, config_id=40)
     inp = wl.make_inputs(w, call=V)
-    out = run_verify(ersd, inp)
-    check_verify(inp, out)
+    for threads in (128, 256):
+        out = run_verify(ersd, inp, block_threads=threads)
+        check_verify(inp, out)
 
 
+@pytest.mark.parametrize("threads", [128, 256])
+@pytest.mark.parametrize("name,scale", [("c1", {}), ("c2", {}), ("c3", dict(B=2)), ("c4", dict(B=2)), ("c5", dict(B=3))])
+def test_both_block_sizes_on_every_configuration(ersd, threads, name, scale):
+    """The kernel is built for 128- and 256-thread blocks and picks one by the number of rows;
+    here each is forced on every configuration (reduced batch)."""
+    inp = wl.make_inputs(wl.scaled(wl.CONFIGS[name], **scale), call=7)
+    for split in (0, 3):
+        check_verify(inp, run_verify(ersd, inp, block_threads=threads, split_v=split))
+
+
+def test_block_size_argument_is_checked(ersd):
+    inp = to_dev(wl.make_inputs(wl.scaled(wl.CONFIGS["c2"], B=1)))
+    tok = torch.empty(1, 5, dtype=torch.int32, device="cuda")
+    acc = torch.empty(1, dtype=torch.int32, device="cuda")
+    with pytest.raises(ersd.ErsdError) as e:
+        ersd.ersd_verify(inp["target"], inp["draft"], inp["seeds"], 1.0, tok, acc, ersd.make_opts(block_threads=96))
+    assert e.value.status == -1
+
+
+@pytest.mark.parametrize("threads", [128, 256])
 @pytest.mark.parametrize("split", [1, 2, 3, 7, 32])
-def test_rows_split_over_several_blocks(ersd, split):
+def test_rows_split_over_several_blocks(ersd, split, threads):
     w = wl.Workload("split", B=2, k=3, V=70001, dtype="bf16", sigma=1.0, T=1.0, config_id=41)
     inp = wl.make_inputs(w)
-    out = run_verify(ersd, inp, split_v=split)
+    out = run_verify(ersd, inp, split_v=split, block_threads=threads)
     check_verify(inp, out)
     t = wl.Workload("split_tree", B=2, k=8, V=40000, dtype="bf16", sigma=1.0, T=1.0, config_id=42,
                     parent=wl.TREE_SPECINFER)
