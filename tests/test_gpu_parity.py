@@ -512,6 +512,27 @@ def test_caller_owned_workspace_and_repeats(ersd):
     assert e.value.status == -5
 
 
+def test_repeated_full_vocabulary_calls_agree_bit_for_bit(ersd):
+    """Stress of the fused finish and of the threshold hand-down: block order varies from launch to
+    launch, results must not (both block sizes, several splits, 40 launches each way)."""
+    w = wl.scaled(wl.CONFIGS["c5"], B=24)
+    inp = to_dev(wl.make_inputs(w, call=3))
+    t = inp["temps"]
+    first = None
+    for threads in (128, 256):
+        for split in (0, 1, 4):
+            o = ersd.make_opts(temps=t, temp_strides=(t.stride(0), t.stride(1)), split_v=split,
+                               block_threads=threads)
+            for rep in range(7):
+                tok = torch.full((w.B, w.k + 1), -7, dtype=torch.int32, device="cuda")
+                acc = torch.full((w.B,), -7, dtype=torch.int32, device="cuda")
+                ersd.ersd_verify(inp["target"], inp["draft"], inp["seeds"], 1.0, tok, acc, o)
+                if first is None:
+                    first = (tok.clone(), acc.clone())
+                assert (tok == first[0]).all() and (acc == first[1]).all(), (threads, split, rep)
+    torch.cuda.synchronize()
+
+
 def test_workspace_reused_by_calls_of_different_sizes(ersd):
     """A small call leaves partial lists behind; a larger call on the same workspace must not
     mistake them for arrival counters (and the other way round)."""
