@@ -212,6 +212,7 @@ def main():
     ap.add_argument("--cpu-seqs", type=int, default=0, help="sequences of the oracle sample (cpu_baseline); 0 = all")
     ap.add_argument("--cpu-passes", type=int, default=8, help="passes of the oracle over its sample (cpu_baseline)")
     ap.add_argument("--split", type=int, default=0, help="thread blocks per row (0: library default)")
+    ap.add_argument("--threads", type=int, default=0, help="threads per block of the kernel (0: library default)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--sigma", type=float, default=None)
@@ -250,7 +251,7 @@ def main():
     stream = torch.cuda.current_stream()
 
     def opts_for(inp):
-        kw = dict(split_v=args.split)
+        kw = dict(split_v=args.split, block_threads=args.threads)
         if inp.get("temps") is not None:
             kw.update(temps=inp["temps"], temp_strides=(inp["temps"].stride(0), inp["temps"].stride(1)))
         return binding.make_opts(**kw)
