@@ -607,6 +607,6 @@ const char* ersd_status_string(int status) {
 
 int ersd_last_cuda_error(void) { return g_last_cuda_error; }
 
-int ersd_version(void) { return 103; }
+int ersd_version(void) { return 104; }
 
 }  // extern "C"
