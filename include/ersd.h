@@ -101,6 +101,11 @@ typedef struct ersd_opts {
   float* out_key;          /* device, nullable, ersd_race_sample: [B, R, c] keys of the arrivals */
   void* workspace;         /* device scratch or NULL (library-owned) */
   size_t workspace_bytes;
+  uint32_t sample_path;    /* ersd_race_sample: 0 = chosen by the library, 1 = the streaming kernel,
+                              2 = the cluster kernel (one thread-block cluster per row, for calls of
+                              few rows; ERSD_EUNSUPPORTED where it does not apply: top_c > 1, rows not
+                              16-byte aligned, B or R > 65535, V > 2^28) */
+  uint32_t reserved1;
 } ersd_opts;
 
 /*

@@ -38,6 +38,7 @@ class ErsdOpts(C.Structure):
         ("out_target_tok", C.c_void_p), ("out_target_key", C.c_void_p),
         ("out_path", C.c_void_p), ("out_key", C.c_void_p),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+        ("sample_path", C.c_uint32), ("reserved1", C.c_uint32),
     ]
 
 
@@ -116,14 +117,26 @@ def _dev(t: torch.Tensor, dtype, name: str):
     return t
 
 
+def _sizes(logits: torch.Tensor, V: Optional[int]):
+    """(B, rows, V) of a logits tensor [B, rows, ld]; V defaults to ld (rows without padding)."""
+    B, rows, ld = logits.shape
+    if V is None:
+        return B, rows, ld
+    if not 1 <= int(V) <= ld:
+        raise ValueError("V must be between 1 and the row length of the tensor")
+    return B, rows, int(V)
+
+
 def make_opts(*, top_c: int = 0, split_v: int = 0, block_threads: int = 0, ld_target: int = 0, ld_draft: int = 0,
               temps: Optional[torch.Tensor] = None, temp_strides: Sequence[int] = (0, 0),
               seq_ids: Optional[torch.Tensor] = None, pos_offsets: Optional[torch.Tensor] = None,
               out_draft_tok=None, out_draft_key=None, out_target_tok=None, out_target_key=None,
-              out_path=None, out_key=None, workspace: Optional[torch.Tensor] = None) -> ErsdOpts:
+              out_path=None, out_key=None, workspace: Optional[torch.Tensor] = None,
+              sample_path: int = 0) -> ErsdOpts:
     o = ErsdOpts()
     o.struct_size = C.sizeof(ErsdOpts)
     o.top_c, o.split_v, o.block_threads = top_c, split_v, block_threads
+    o.sample_path = sample_path
     o.ld_target, o.ld_draft = ld_target, ld_draft
     if temps is not None:
         _dev(temps, torch.float32, "temps")
@@ -175,12 +188,13 @@ def ersd_optimal_tree(accept: Sequence[float], k: int):
 
 
 def ersd_race_sample(logits: torch.Tensor, seeds: torch.Tensor, T: float, out_tok: torch.Tensor,
-                     opts: Optional[ErsdOpts] = None, stream=None) -> None:
-    """logits [B, R, V] (f32/bf16), seeds int64 [B] (the uint64 bit patterns), out_tok int32 [B, R, c]."""
+                     opts: Optional[ErsdOpts] = None, stream=None, V: Optional[int] = None) -> None:
+    """logits [B, R, V] (f32/bf16), seeds int64 [B] (the uint64 bit patterns), out_tok int32 [B, R, c].
+    Padded rows: pass the tensor [B, R, ld], the vocabulary size as ``V`` and opts.ld_target = ld."""
     _dev(logits, None, "logits")
     _dev(seeds, torch.int64, "seeds")
     _dev(out_tok, torch.int32, "out_tok")
-    B, R, V = logits.shape
+    B, R, V = _sizes(logits, V)
     _check(lib().ersd_race_sample(_ptr(logits), _dtype_code(logits), _ptr(seeds), B, R, V, float(T),
                                   _ptr(out_tok), C.byref(opts) if opts is not None else None,
                                   _stream(stream)), "ersd_race_sample")
@@ -188,10 +202,11 @@ def ersd_race_sample(logits: torch.Tensor, seeds: torch.Tensor, T: float, out_to
 
 def ersd_verify(target_logits: torch.Tensor, draft_logits: Optional[torch.Tensor], seeds: torch.Tensor,
                 T: float, out_tokens: torch.Tensor, out_accept_len: torch.Tensor,
-                opts: Optional[ErsdOpts] = None, stream=None) -> None:
-    """target [B, k+1, V], draft [B, k, V], out_tokens int32 [B, k+1], out_accept_len int32 [B]."""
+                opts: Optional[ErsdOpts] = None, stream=None, V: Optional[int] = None) -> None:
+    """target [B, k+1, V], draft [B, k, V], out_tokens int32 [B, k+1], out_accept_len int32 [B].
+    Padded rows: tensors [B, rows, ld], the vocabulary size as ``V``, opts.ld_target / ld_draft = ld."""
     _dev(target_logits, None, "target_logits")
-    B, rows, V = target_logits.shape
+    B, rows, V = _sizes(target_logits, V)
     if draft_logits is not None:
         _dev(draft_logits, target_logits.dtype, "draft_logits")
     _dev(seeds, torch.int64, "seeds")
@@ -205,11 +220,11 @@ def ersd_verify(target_logits: torch.Tensor, draft_logits: Optional[torch.Tensor
 
 def ersd_verify_tokens(target_logits: torch.Tensor, draft_tokens: Optional[torch.Tensor], seeds: torch.Tensor,
                        T: float, out_tokens: torch.Tensor, out_accept_len: torch.Tensor,
-                       opts: Optional[ErsdOpts] = None, stream=None) -> None:
+                       opts: Optional[ErsdOpts] = None, stream=None, V: Optional[int] = None) -> None:
     """target [B, k+1, V], draft_tokens int32 [B, k] (drafted earlier with the same races),
     out_tokens int32 [B, k+1], out_accept_len int32 [B]."""
     _dev(target_logits, None, "target_logits")
-    B, rows, V = target_logits.shape
+    B, rows, V = _sizes(target_logits, V)
     if draft_tokens is not None:
         _dev(draft_tokens, torch.int32, "draft_tokens")
     _dev(seeds, torch.int64, "seeds")
@@ -223,12 +238,13 @@ def ersd_verify_tokens(target_logits: torch.Tensor, draft_tokens: Optional[torch
 
 def ersd_verify_noalloc(target_logits: torch.Tensor, draft_logits: Optional[torch.Tensor],
                         seeds: torch.Tensor, T: float, out_tokens: torch.Tensor,
-                        out_accept_len: torch.Tensor, opts: Optional[ErsdOpts] = None, stream=None) -> None:
+                        out_accept_len: torch.Tensor, opts: Optional[ErsdOpts] = None, stream=None,
+                        V: Optional[int] = None) -> None:
     """ersd_verify for callers that cannot allocate device memory: same arguments and results,
     scratch built into the library, B * (k + 1) <= ERSD_NOALLOC_MAX_ROWS.  Calls on one device
     share that scratch, so they must not overlap on the GPU."""
     _dev(target_logits, None, "target_logits")
-    B, rows, V = target_logits.shape
+    B, rows, V = _sizes(target_logits, V)
     if draft_logits is not None:
         _dev(draft_logits, target_logits.dtype, "draft_logits")
     _dev(seeds, torch.int64, "seeds")
@@ -242,10 +258,11 @@ def ersd_verify_noalloc(target_logits: torch.Tensor, draft_logits: Optional[torc
 
 def ersd_verify_tree(target_logits: torch.Tensor, draft_logits: Optional[torch.Tensor],
                      parent: Sequence[int], seeds: torch.Tensor, T: float, out_tokens: torch.Tensor,
-                     out_accept_len: torch.Tensor, opts: Optional[ErsdOpts] = None, stream=None) -> None:
+                     out_accept_len: torch.Tensor, opts: Optional[ErsdOpts] = None, stream=None,
+                     V: Optional[int] = None) -> None:
     """target, draft [B, N+1, V]; parent: host list [N+1]; out_tokens int32 [B, D+1]."""
     _dev(target_logits, None, "target_logits")
-    B, nodes, V = target_logits.shape
+    B, nodes, V = _sizes(target_logits, V)
     if draft_logits is not None:
         _dev(draft_logits, target_logits.dtype, "draft_logits")
     _dev(seeds, torch.int64, "seeds")

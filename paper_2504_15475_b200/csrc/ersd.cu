@@ -98,6 +98,9 @@ namespace b128 {
 constexpr int kThreads = 128, kMinBlocks = 8;
 #include "ersd_kernel.inc"
 }  // namespace b128
+namespace b256 {
+#include "ersd_cluster.inc"
+}  // namespace b256
 
 template <int DT>
 __global__ void ersd_row_keys_kernel(const void* row, int V, float T, uint64_t seed, uint32_t seq,
@@ -330,6 +333,87 @@ static int launch(const Params& p, const TreeDesc& tree, int dt, cudaStream_t st
   return e == cudaSuccess ? ERSD_OK : cuda_fail(e);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Latency path of ersd_race_sample: one cluster of thread blocks per row (ersd_cluster.inc).
+// ---------------------------------------------------------------------------------------------
+constexpr int64_t kClusterAutoUnits = 24;  // default: rows per call up to which the cluster kernel is taken
+
+// Largest cluster (a power of two) the device takes for the cluster kernels: 16 where the opt-in
+// for non-portable sizes is granted and such a cluster fits, else 8.  Asked once per device.
+static int cluster_limit(int* out) {
+  static std::mutex m;
+  static int limit[64];
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (dev < 0 || dev >= 64) return ERSD_EUNSUPPORTED;
+  std::lock_guard<std::mutex> lock(m);
+  if (!limit[dev]) {
+    const void* kernels[2] = {(const void*)b256::ersd_sample_cluster_kernel<ERSD_BF16>,
+                              (const void*)b256::ersd_sample_cluster_kernel<ERSD_F32>};
+    int lim = 16;
+    for (int q = 0; q < 2 && lim == 16; ++q) {
+      e = cudaFuncSetAttribute(kernels[q], cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+      int n = 0;
+      if (e == cudaSuccess) {
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof cfg);
+        cfg.gridDim = dim3(16, 1, 1);
+        cfg.blockDim = dim3(b256::kThreads, 1, 1);
+        cudaLaunchAttribute at;
+        at.id = cudaLaunchAttributeClusterDimension;
+        at.val.clusterDim.x = 16;
+        at.val.clusterDim.y = 1;
+        at.val.clusterDim.z = 1;
+        cfg.attrs = &at;
+        cfg.numAttrs = 1;
+        e = cudaOccupancyMaxActiveClusters(&n, kernels[q], &cfg);
+      }
+      if (e != cudaSuccess || n < 1) lim = 8;
+    }
+    (void)cudaGetLastError();  // a refused opt-in only means clusters of eight
+    limit[dev] = lim;
+  }
+  *out = limit[dev];
+  return ERSD_OK;
+}
+
+// Whether a sampling call can take the cluster kernel at all.
+static bool cluster_applies(const Params& p) {
+  return p.c_sample == 1 && p.aligned_t && p.rows <= 65535 && p.B <= 65535 && p.V <= (1 << 28);
+}
+
+template <int DT>
+static int launch_cluster_dt(const Params& p, cudaStream_t st) {
+  auto kernel = b256::ersd_sample_cluster_kernel<DT>;
+  int lim = 8;
+  const int ls = cluster_limit(&lim);
+  if (ls != ERSD_OK) return ls;
+  // smallest power of two that lets a thread hold its share of the row in registers at once
+  const int ntiles = (p.V + b256::kTile - 1) / b256::kTile;
+  int CL = 1;
+  while (CL < lim && CL * b256::kClusterGroups < ntiles) CL *= 2;
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3((unsigned)CL, (unsigned)p.rows, (unsigned)p.B);
+  cfg.blockDim = dim3(b256::kThreads, 1, 1);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute at;
+  at.id = cudaLaunchAttributeClusterDimension;
+  at.val.clusterDim.x = (unsigned)CL;
+  at.val.clusterDim.y = 1;
+  at.val.clusterDim.z = 1;
+  cfg.attrs = &at;
+  cfg.numAttrs = 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, p);
+  return e == cudaSuccess ? ERSD_OK : cuda_fail(e);
+}
+
+static int launch_cluster(const Params& p, int dt, cudaStream_t st) {
+  return dt == ERSD_BF16 ? launch_cluster_dt<ERSD_BF16>(p, st) : launch_cluster_dt<ERSD_F32>(p, st);
+}
+
 static int check_common(const void* logits, int dt, const uint64_t* seeds, int B, int rows, int V,
                         float T) {
   if (!logits || !seeds) return ERSD_EINVAL;
@@ -450,6 +534,11 @@ int ersd_race_sample(const void* logits, ersd_dtype dt, const uint64_t* seeds, i
   p.aligned_d = 1;
   p.out_tokens = out_tok;
   p.out_key = o.out_key;
+  if (o.sample_path > 2) return ERSD_EINVAL;
+  if (o.sample_path == 2 && !cluster_applies(p)) return ERSD_EUNSUPPORTED;
+  if (o.sample_path == 2 || (o.sample_path == 0 && o.split_v == 0 && o.block_threads == 0 &&
+                             (int64_t)B * R <= kClusterAutoUnits && cluster_applies(p)))
+    return launch_cluster(p, dt, (cudaStream_t)cuda_stream);
   st = choose_threads(o, (int64_t)B * R, &p.threads);
   if (st != ERSD_OK) return st;
   set_chunks(p, choose_split(o, (int64_t)B * R, V, c, p.threads));

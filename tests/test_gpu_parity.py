@@ -208,11 +208,13 @@ def test_row_strides_and_unaligned_rows(ersd):
     for dtype in (torch.float32, torch.bfloat16):
         big_t = (torch.randn(B, k + 1, ld, generator=g) * 2).to(dtype)
         big_d = (torch.randn(B, k, ld, generator=g) * 2).to(dtype)
+        big_t[:, :, V:] = 50.0                # the padding must never be raced
+        big_d[:, :, V:] = 50.0
         seeds = wl.make_seeds(1, 2, B)
         opts = ersd.make_opts(ld_target=ld, ld_draft=ld)
         tok = torch.empty(B, k + 1, dtype=torch.int32, device="cuda")
         acc = torch.empty(B, dtype=torch.int32, device="cuda")
-        ersd.ersd_verify(big_t.cuda(), big_d.cuda(), seeds.cuda(), 1.0, tok, acc, opts)
+        ersd.ersd_verify(big_t.cuda(), big_d.cuda(), seeds.cuda(), 1.0, tok, acc, opts, V=V)
         torch.cuda.synchronize()
         import oracle
         ref = oracle.verify(wl.as_numpy_logits(big_t[:, :, :V].contiguous()),
@@ -236,12 +238,14 @@ def test_padded_rows_on_the_vector_path_and_many_small_sequences(ersd):
     g = torch.Generator().manual_seed(21)
     big_t = (torch.randn(B, k + 1, ld, generator=g) * 2).to(torch.bfloat16)
     big_d = (torch.randn(B, k, ld, generator=g) * 2).to(torch.bfloat16)
+    big_t[:, :, V:] = 50.0                    # the padding must never be raced
+    big_d[:, :, V:] = 50.0
     seeds = wl.make_seeds(9, 1, B)
     tok = torch.empty(B, k + 1, dtype=torch.int32, device="cuda")
     acc = torch.empty(B, dtype=torch.int32, device="cuda")
     for split in (0, 2):
         ersd.ersd_verify(big_t.cuda(), big_d.cuda(), seeds.cuda(), 0.8, tok, acc,
-                         ersd.make_opts(ld_target=ld, ld_draft=ld, split_v=split))
+                         ersd.make_opts(ld_target=ld, ld_draft=ld, split_v=split), V=V)
         torch.cuda.synchronize()
         ref = oracle.verify(wl.as_numpy_logits(big_t[:, :, :V].contiguous()),
                             wl.as_numpy_logits(big_d[:, :, :V].contiguous()), wl.seeds_as_u64(seeds), T=0.8)
@@ -276,6 +280,33 @@ def test_special_values(ersd):
         assert tok[0, 0] == -1 and out["accept_len"][0].item() == 0
         assert out["draft_tok"][1, 0].item() == 17
         assert tok[2, 0] == 123 and out["accept_len"][2].item() == 1
+
+
+@pytest.mark.parametrize("threads", [128, 256])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_infinite_logits_far_into_the_row(ersd, dtype, threads):
+    """+inf at even and odd positions beyond the first tile (where groups of eight logits are
+    ruled out by their maximum alone): such a token always wins, the lowest index first."""
+    V = 40000
+    g = torch.Generator().manual_seed(19)
+    t = torch.randn(4, 2, V, generator=g)
+    d = torch.randn(4, 1, V, generator=g)
+    t[0, 0, 30001] = float("inf")
+    d[0, 0, 22222] = float("inf")
+    t[1, 0, 39999] = float("inf")
+    t[1, 0, 17001] = float("inf")
+    d[1, 0, 17001] = float("inf")
+    t[2, 0, 9000:] = float("-inf")                   # a masked range ...
+    t[2, 0, 33333] = float("inf")                    # ... with one infinite logit inside
+    d[2, 0, 1::2] = float("-inf")                    # every odd position masked
+    t[3, 1, 2049] = float("inf")
+    inp = dict(target=wl._storage(t, dtype), draft=wl._storage(d, dtype), seeds=wl.make_seeds(4, 0, 4),
+               T=0.8, temps=None, parent=None)
+    out = run_verify(ersd, inp, block_threads=threads)
+    check_verify(inp, out)
+    assert out["target_tok"][:, 0].cpu().tolist()[:3] == [30001, 17001, 33333]
+    assert out["draft_tok"][:2, 0].cpu().tolist() == [22222, 17001]
+    assert out["target_tok"][3, 1].item() == 2049 and out["draft_tok"][2, 0].item() % 2 == 0
 
 
 def test_greedy_temperature_zero(ersd):
