@@ -104,7 +104,7 @@ typedef struct ersd_opts {
   uint32_t sample_path;    /* ersd_race_sample: 0 = chosen by the library, 1 = the streaming kernel,
                               2 = the cluster kernel (one thread-block cluster per row, for calls of
                               few rows; ERSD_EUNSUPPORTED where it does not apply: top_c > 1, rows not
-                              16-byte aligned, B or R > 65535, V > 2^28) */
+                              16-byte aligned, B or R > 65535, V > 327680) */
   uint32_t reserved1;
 } ersd_opts;
 

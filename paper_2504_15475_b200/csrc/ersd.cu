@@ -336,7 +336,8 @@ static int launch(const Params& p, const TreeDesc& tree, int dt, cudaStream_t st
 // ---------------------------------------------------------------------------------------------
 // Latency path of ersd_race_sample: one cluster of thread blocks per row (ersd_cluster.inc).
 // ---------------------------------------------------------------------------------------------
-constexpr int64_t kClusterAutoUnits = 24;  // default: rows per call up to which the cluster kernel is taken
+constexpr int64_t kClusterAutoUnits = 64;
+constexpr int kClusterMaxTiles = 20;  // tiles a block of the cluster kernel can stage (180 KB of fp32 logits)  // default: rows per call up to which the cluster kernel is taken
 
 // Largest cluster (a power of two) the device takes for the cluster kernels: 16 where the opt-in
 // for non-portable sizes is granted and such a cluster fits, else 8.  Asked once per device.
@@ -351,7 +352,13 @@ static int cluster_limit(int* out) {
   if (!limit[dev]) {
     const void* kernels[2] = {(const void*)b256::ersd_sample_cluster_kernel<ERSD_BF16>,
                               (const void*)b256::ersd_sample_cluster_kernel<ERSD_F32>};
+    const int smem[2] = {(int)b256::cluster_smem_bytes<ERSD_BF16>(kClusterMaxTiles),
+                         (int)b256::cluster_smem_bytes<ERSD_F32>(kClusterMaxTiles)};
     int lim = 16;
+    for (int q = 0; q < 2; ++q) {
+      e = cudaFuncSetAttribute(kernels[q], cudaFuncAttributeMaxDynamicSharedMemorySize, smem[q]);
+      if (e != cudaSuccess) return cuda_fail(e);
+    }
     for (int q = 0; q < 2 && lim == 16; ++q) {
       e = cudaFuncSetAttribute(kernels[q], cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
       int n = 0;
@@ -360,6 +367,7 @@ static int cluster_limit(int* out) {
         memset(&cfg, 0, sizeof cfg);
         cfg.gridDim = dim3(16, 1, 1);
         cfg.blockDim = dim3(b256::kThreads, 1, 1);
+        cfg.dynamicSmemBytes = (size_t)smem[q];
         cudaLaunchAttribute at;
         at.id = cudaLaunchAttributeClusterDimension;
         at.val.clusterDim.x = 16;
@@ -380,7 +388,9 @@ static int cluster_limit(int* out) {
 
 // Whether a sampling call can take the cluster kernel at all.
 static bool cluster_applies(const Params& p) {
-  return p.c_sample == 1 && p.aligned_t && p.rows <= 65535 && p.B <= 65535 && p.V <= (1 << 28);
+  // (eight blocks, the portable cluster size, must be able to stage the row)
+  return p.c_sample == 1 && p.aligned_t && p.rows <= 65535 && p.B <= 65535 &&
+         p.V <= 8 * kClusterMaxTiles * b256::kTile;
 }
 
 template <int DT>
@@ -393,11 +403,12 @@ static int launch_cluster_dt(const Params& p, cudaStream_t st) {
   const int ntiles = (p.V + b256::kTile - 1) / b256::kTile;
   int CL = 1;
   while (CL < lim && CL * b256::kClusterGroups < ntiles) CL *= 2;
+  const int G = (ntiles + CL - 1) / CL;  // tiles per block; at most kClusterMaxTiles, see cluster_applies
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
   cfg.gridDim = dim3((unsigned)CL, (unsigned)p.rows, (unsigned)p.B);
   cfg.blockDim = dim3(b256::kThreads, 1, 1);
-  cfg.dynamicSmemBytes = 0;
+  cfg.dynamicSmemBytes = b256::cluster_smem_bytes<DT>(G);
   cfg.stream = st;
   cudaLaunchAttribute at;
   at.id = cudaLaunchAttributeClusterDimension;

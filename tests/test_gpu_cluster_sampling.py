@@ -212,3 +212,26 @@ def test_repeated_calls_agree_bit_for_bit(ersd):
         else:
             assert (tok == first[0]).all() and (key == first[1]).all()
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("gap", [1e-4, -1e-4, 3e-3, -3e-3])
+def test_screening_keys_too_close_to_call_are_decided_exactly(ersd, gap):
+    """Two tokens whose keys differ by less than the screening precision (about 1.4e-3) but by
+    far more than the near-tie window: the exact key must decide, whichever of the two leads."""
+    import oracle
+    B, V, T = 6, 128256, 1.0
+    seeds = wl.make_seeds(31, 0, B)
+    flat = np.zeros((B, 1, V), dtype=np.float32)
+    tok2, key2 = oracle.race_sample(flat, wl.seeds_as_u64(seeds), T=T, c=2)
+    logits = torch.zeros(B, 1, V, dtype=torch.float32)
+    want = []
+    for b in range(B):
+        first, second = int(tok2[b, 0, 0]), int(tok2[b, 0, 1])
+        # raise the runner-up's logit until its key sits `gap` above (or below) the leader's
+        logits[b, 0, second] = float((key2[b, 0, 1] - key2[b, 0, 0] - gap) * T)
+        want.append(first if gap > 0 else second)
+    tok, key = sample(ersd, logits, seeds, T, CLUSTER)
+    assert check_sample(logits, seeds, T, tok, key) == 0
+    assert tok[:, 0, 0].cpu().tolist() == want
+    tok_s, key_s = sample(ersd, logits, seeds, T, STREAMING)
+    assert (tok == tok_s).all() and (key == key_s).all()
