@@ -336,7 +336,7 @@ static int launch(const Params& p, const TreeDesc& tree, int dt, cudaStream_t st
 // ---------------------------------------------------------------------------------------------
 // Latency path of ersd_race_sample: one cluster of thread blocks per row (ersd_cluster.inc).
 // ---------------------------------------------------------------------------------------------
-constexpr int64_t kClusterAutoUnits = 64;
+constexpr int64_t kClusterAutoUnits = 96;
 constexpr int kClusterMaxTiles = 20;  // tiles a block of the cluster kernel can stage (180 KB of fp32 logits)  // default: rows per call up to which the cluster kernel is taken
 
 // Largest cluster (a power of two) the device takes for the cluster kernels: 16 where the opt-in
