@@ -38,7 +38,7 @@ class ErsdOpts(C.Structure):
         ("out_target_tok", C.c_void_p), ("out_target_key", C.c_void_p),
         ("out_path", C.c_void_p), ("out_key", C.c_void_p),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
-        ("sample_path", C.c_uint32), ("reserved1", C.c_uint32),
+        ("kernel_path", C.c_uint32), ("reserved1", C.c_uint32),
     ]
 
 
@@ -132,11 +132,11 @@ def make_opts(*, top_c: int = 0, split_v: int = 0, block_threads: int = 0, ld_ta
               seq_ids: Optional[torch.Tensor] = None, pos_offsets: Optional[torch.Tensor] = None,
               out_draft_tok=None, out_draft_key=None, out_target_tok=None, out_target_key=None,
               out_path=None, out_key=None, workspace: Optional[torch.Tensor] = None,
-              sample_path: int = 0) -> ErsdOpts:
+              kernel_path: int = 0) -> ErsdOpts:
     o = ErsdOpts()
     o.struct_size = C.sizeof(ErsdOpts)
     o.top_c, o.split_v, o.block_threads = top_c, split_v, block_threads
-    o.sample_path = sample_path
+    o.kernel_path = kernel_path
     o.ld_target, o.ld_draft = ld_target, ld_draft
     if temps is not None:
         _dev(temps, torch.float32, "temps")
@@ -286,14 +286,15 @@ def ersd_row_keys(row: torch.Tensor, T: float, seed: int, seq_id: int, position:
 
 # --------------------------------------------------------------------------- conveniences
 def verify(target_logits, draft_logits, seeds, T=1.0, temps=None, parent=None, split_v=0,
-           want_rows=False, seq_ids=None, pos_offsets=None, block_threads=0):
+           want_rows=False, seq_ids=None, pos_offsets=None, block_threads=0, kernel_path=0):
     """Allocate outputs, call ersd_verify / ersd_verify_tree, return a dict of device tensors."""
     B, rows, V = target_logits.shape
     dev = target_logits.device
     D = rows - 1 if parent is None else ersd_tree_depth(parent)
     out = dict(tokens=torch.empty(B, D + 1, dtype=torch.int32, device=dev),
                accept_len=torch.empty(B, dtype=torch.int32, device=dev))
-    kw = dict(split_v=split_v, block_threads=block_threads, seq_ids=seq_ids, pos_offsets=pos_offsets)
+    kw = dict(split_v=split_v, block_threads=block_threads, seq_ids=seq_ids, pos_offsets=pos_offsets,
+              kernel_path=kernel_path)
     if temps is not None:
         kw.update(temps=temps, temp_strides=(temps.stride(0), temps.stride(1)))
     if want_rows:

@@ -337,7 +337,13 @@ static int launch(const Params& p, const TreeDesc& tree, int dt, cudaStream_t st
 // Latency path of ersd_race_sample: one cluster of thread blocks per row (ersd_cluster.inc).
 // ---------------------------------------------------------------------------------------------
 constexpr int64_t kClusterAutoUnits = 96;
-constexpr int kClusterMaxTiles = 20;  // tiles a block of the cluster kernel can stage (180 KB of fp32 logits)  // default: rows per call up to which the cluster kernel is taken
+constexpr size_t kClusterSmemBytes = 200 * 1024;  // dynamic shared memory a block of the cluster kernel may use
+
+// Tiles per block that fit (roles = rows raced together: 1, or 2 for a draft/target pair).
+static int cluster_max_tiles(int dt, int roles) {
+  const size_t per_tile = dt == ERSD_BF16 ? b256::cluster_role_bytes<ERSD_BF16>(1) : b256::cluster_role_bytes<ERSD_F32>(1);
+  return (int)(kClusterSmemBytes / (per_tile * (size_t)roles));
+}  // default: rows per call up to which the cluster kernel is taken
 
 // Largest cluster (a power of two) the device takes for the cluster kernels: 16 where the opt-in
 // for non-portable sizes is granted and such a cluster fits, else 8.  Asked once per device.
@@ -350,10 +356,9 @@ static int cluster_limit(int* out) {
   if (dev < 0 || dev >= 64) return ERSD_EUNSUPPORTED;
   std::lock_guard<std::mutex> lock(m);
   if (!limit[dev]) {
-    const void* kernels[2] = {(const void*)b256::ersd_sample_cluster_kernel<ERSD_BF16>,
-                              (const void*)b256::ersd_sample_cluster_kernel<ERSD_F32>};
-    const int smem[2] = {(int)b256::cluster_smem_bytes<ERSD_BF16>(kClusterMaxTiles),
-                         (int)b256::cluster_smem_bytes<ERSD_F32>(kClusterMaxTiles)};
+    const void* kernels[2] = {(const void*)b256::ersd_cluster_kernel<ERSD_BF16>,
+                              (const void*)b256::ersd_cluster_kernel<ERSD_F32>};
+    const int smem[2] = {(int)kClusterSmemBytes, (int)kClusterSmemBytes};
     int lim = 16;
     for (int q = 0; q < 2; ++q) {
       e = cudaFuncSetAttribute(kernels[q], cudaFuncAttributeMaxDynamicSharedMemorySize, smem[q]);
@@ -387,15 +392,18 @@ static int cluster_limit(int* out) {
 }
 
 // Whether a sampling call can take the cluster kernel at all.
-static bool cluster_applies(const Params& p) {
-  // (eight blocks, the portable cluster size, must be able to stage the row)
-  return p.c_sample == 1 && p.aligned_t && p.rows <= 65535 && p.B <= 65535 &&
-         p.V <= 8 * kClusterMaxTiles * b256::kTile;
+static bool cluster_applies(const Params& p, int dt) {
+  // (eight blocks, the portable cluster size, must be able to stage the rows of a position)
+  const int roles = (p.mode == kVerify && p.draft) ? 2 : 1;
+  const int64_t ntiles = ((int64_t)p.V + b256::kTile - 1) / b256::kTile;
+  if (ntiles > 8 * (int64_t)cluster_max_tiles(dt, roles)) return false;
+  if (p.mode == kVerify && p.rows > 32) return false;
+  return p.c_sample == 1 && p.aligned_t && (roles == 1 || p.aligned_d) && p.rows <= 65535 && p.B <= 65535;
 }
 
 template <int DT>
 static int launch_cluster_dt(const Params& p, cudaStream_t st) {
-  auto kernel = b256::ersd_sample_cluster_kernel<DT>;
+  auto kernel = b256::ersd_cluster_kernel<DT>;
   int lim = 8;
   const int ls = cluster_limit(&lim);
   if (ls != ERSD_OK) return ls;
@@ -403,12 +411,13 @@ static int launch_cluster_dt(const Params& p, cudaStream_t st) {
   const int ntiles = (p.V + b256::kTile - 1) / b256::kTile;
   int CL = 1;
   while (CL < lim && CL * b256::kClusterGroups < ntiles) CL *= 2;
-  const int G = (ntiles + CL - 1) / CL;  // tiles per block; at most kClusterMaxTiles, see cluster_applies
+  const int G = (ntiles + CL - 1) / CL;  // tiles per block; they fit, see cluster_applies
+  const int roles = (p.mode == kVerify && p.draft) ? 2 : 1;
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
   cfg.gridDim = dim3((unsigned)CL, (unsigned)p.rows, (unsigned)p.B);
   cfg.blockDim = dim3(b256::kThreads, 1, 1);
-  cfg.dynamicSmemBytes = b256::cluster_smem_bytes<DT>(G);
+  cfg.dynamicSmemBytes = b256::cluster_role_bytes<DT>(G) * (size_t)roles;
   cfg.stream = st;
   cudaLaunchAttribute at;
   at.id = cudaLaunchAttributeClusterDimension;
@@ -480,13 +489,20 @@ static int verify_impl(const void* target, const void* draft, int dt, const Tree
   p.out_draft_key = o.out_draft_key;
   p.out_target_tok = o.out_target_tok;
   p.out_target_key = o.out_target_key;
-  int st0 = choose_threads(o, (int64_t)B * rows, &p.threads);
-  if (st0 != ERSD_OK) return st0;
-  set_chunks(p, choose_split(o, (int64_t)B * rows, V, cmax, p.threads));
   void* ws = nullptr;
   const int st = get_workspace(o, workspace_bytes(B, rows), &ws);
   if (st != ERSD_OK) return st;
   p.slots = (Slot*)ws;
+  // sequences of few rows: one cluster per position (chains only: one arrival per race)
+  if (o.kernel_path > 2) return ERSD_EINVAL;
+  const bool cluster_ok = chain && cmax <= 1 && cluster_applies(p, dt);
+  if (o.kernel_path == 2 && !cluster_ok) return ERSD_EUNSUPPORTED;
+  if (o.kernel_path == 2 || (o.kernel_path == 0 && o.split_v == 0 && o.block_threads == 0 &&
+                             (int64_t)B * rows <= kClusterAutoUnits && cluster_ok))
+    return launch_cluster(p, dt, (cudaStream_t)stream);
+  int st0 = choose_threads(o, (int64_t)B * rows, &p.threads);
+  if (st0 != ERSD_OK) return st0;
+  set_chunks(p, choose_split(o, (int64_t)B * rows, V, cmax, p.threads));
   return launch(p, tree, dt, (cudaStream_t)stream);
 }
 
@@ -545,10 +561,10 @@ int ersd_race_sample(const void* logits, ersd_dtype dt, const uint64_t* seeds, i
   p.aligned_d = 1;
   p.out_tokens = out_tok;
   p.out_key = o.out_key;
-  if (o.sample_path > 2) return ERSD_EINVAL;
-  if (o.sample_path == 2 && !cluster_applies(p)) return ERSD_EUNSUPPORTED;
-  if (o.sample_path == 2 || (o.sample_path == 0 && o.split_v == 0 && o.block_threads == 0 &&
-                             (int64_t)B * R <= kClusterAutoUnits && cluster_applies(p)))
+  if (o.kernel_path > 2) return ERSD_EINVAL;
+  if (o.kernel_path == 2 && !cluster_applies(p, dt)) return ERSD_EUNSUPPORTED;
+  if (o.kernel_path == 2 || (o.kernel_path == 0 && o.split_v == 0 && o.block_threads == 0 &&
+                             (int64_t)B * R <= kClusterAutoUnits && cluster_applies(p, dt)))
     return launch_cluster(p, dt, (cudaStream_t)cuda_stream);
   st = choose_threads(o, (int64_t)B * R, &p.threads);
   if (st != ERSD_OK) return st;

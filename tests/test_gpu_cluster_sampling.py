@@ -1,5 +1,5 @@
 """The latency path of race sampling (one thread-block cluster per logit row) against the CPU
-oracle, through the C boundary.  `sample_path=2` forces the cluster kernel, `1` the streaming one."""
+oracle, through the C boundary.  `kernel_path=2` forces the cluster kernel, `1` the streaming one."""
 import numpy as np
 import pytest
 import torch
@@ -31,7 +31,7 @@ def sample(ersd, logits, seeds, T, path, **kw):
     tok = torch.full((B, R, 1), -7, dtype=torch.int32, device="cuda")
     key = torch.full((B, R, 1), -7.0, dtype=torch.float32, device="cuda")
     ersd.ersd_race_sample(big.cuda(), seeds.cuda(), T, tok,
-                          ersd.make_opts(sample_path=path, out_key=key, ld_target=ld, **kw), V=V)
+                          ersd.make_opts(kernel_path=path, out_key=key, ld_target=ld, **kw), V=V)
     torch.cuda.synchronize()
     return tok, key
 
@@ -126,7 +126,7 @@ def test_per_row_temperatures_sequence_ids_offsets_and_strides(ersd):
     seeds = wl.make_seeds(6, 0, B)
     tok = torch.full((B, R, 1), -7, dtype=torch.int32, device="cuda")
     key = torch.full((B, R, 1), -7.0, dtype=torch.float32, device="cuda")
-    opts = ersd.make_opts(sample_path=CLUSTER, out_key=key, ld_target=ld, temps=temps.cuda(), temp_strides=(R, 1),
+    opts = ersd.make_opts(kernel_path=CLUSTER, out_key=key, ld_target=ld, temps=temps.cuda(), temp_strides=(R, 1),
                           seq_ids=seq.cuda(), pos_offsets=off.cuda())
     ersd.ersd_race_sample(big.cuda(), seeds.cuda(), 1.0, tok, opts, V=V)
     torch.cuda.synchronize()
@@ -136,7 +136,7 @@ def test_per_row_temperatures_sequence_ids_offsets_and_strides(ersd):
     temps_ok[3, 1] = 1.0
     temps_ok[3, 2] = 1.0
     ersd.ersd_race_sample(big.cuda(), seeds.cuda(), 1.0, tok,
-                          ersd.make_opts(sample_path=CLUSTER, out_key=key, ld_target=ld, temps=temps_ok.cuda(),
+                          ersd.make_opts(kernel_path=CLUSTER, out_key=key, ld_target=ld, temps=temps_ok.cuda(),
                                          temp_strides=(R, 1), seq_ids=seq.cuda(), pos_offsets=off.cuda()), V=V)
     torch.cuda.synchronize()
     assert check_sample(logits, seeds, 1.0, tok, key, temps=temps_ok.numpy(),
@@ -149,14 +149,14 @@ def test_where_the_cluster_kernel_does_not_apply(ersd):
     seeds = wl.make_seeds(1, 0, B).cuda()
     tok = torch.empty(B, R, 4, dtype=torch.int32, device="cuda")
     with pytest.raises(ersd.ErsdError) as e:
-        ersd.ersd_race_sample(logits, seeds, 1.0, tok, ersd.make_opts(sample_path=CLUSTER))
+        ersd.ersd_race_sample(logits, seeds, 1.0, tok, ersd.make_opts(kernel_path=CLUSTER))
     assert e.value.status == -3
     ok = torch.randn(B, R, 1024).to(torch.bfloat16).cuda()
     with pytest.raises(ersd.ErsdError) as e:
-        ersd.ersd_race_sample(ok, seeds, 1.0, tok, ersd.make_opts(sample_path=CLUSTER, top_c=4))
+        ersd.ersd_race_sample(ok, seeds, 1.0, tok, ersd.make_opts(kernel_path=CLUSTER, top_c=4))
     assert e.value.status == -3
     with pytest.raises(ersd.ErsdError) as e:
-        ersd.ersd_race_sample(ok, seeds, 1.0, tok, ersd.make_opts(sample_path=3))
+        ersd.ersd_race_sample(ok, seeds, 1.0, tok, ersd.make_opts(kernel_path=3))
     assert e.value.status == -1
     # left to the library, such calls take the streaming kernel
     ersd.ersd_race_sample(logits, seeds, 1.0, tok, ersd.make_opts(top_c=4))
@@ -191,7 +191,7 @@ def test_drafting_loop_one_position_at_a_time(ersd):
         off = torch.full((B,), j, dtype=torch.int32, device="cuda")
         row = dev[:, j:j + 1, :].contiguous()
         tok = torch.empty(B, 1, 1, dtype=torch.int32, device="cuda")
-        ersd.ersd_race_sample(row, seeds.cuda(), 0.7, tok, ersd.make_opts(sample_path=CLUSTER, pos_offsets=off))
+        ersd.ersd_race_sample(row, seeds.cuda(), 0.7, tok, ersd.make_opts(kernel_path=CLUSTER, pos_offsets=off))
         got[:, j] = tok[:, 0]
     torch.cuda.synchronize()
     assert check_sample(logits, seeds, 0.7, got, None) == 0
@@ -206,7 +206,7 @@ def test_repeated_calls_agree_bit_for_bit(ersd):
     for _ in range(50):
         tok = torch.empty(B, 1, 1, dtype=torch.int32, device="cuda")
         key = torch.empty(B, 1, 1, dtype=torch.float32, device="cuda")
-        ersd.ersd_race_sample(logits, seeds, 1.0, tok, ersd.make_opts(sample_path=CLUSTER, out_key=key))
+        ersd.ersd_race_sample(logits, seeds, 1.0, tok, ersd.make_opts(kernel_path=CLUSTER, out_key=key))
         if first is None:
             first = (tok, key)
         else:
