@@ -334,9 +334,12 @@ static int launch(const Params& p, const TreeDesc& tree, int dt, cudaStream_t st
 }
 
 // ---------------------------------------------------------------------------------------------
-// Latency path of ersd_race_sample: one cluster of thread blocks per row (ersd_cluster.inc).
+// Latency path of calls of few rows: one cluster of thread blocks per position (ersd_cluster.inc).
 // ---------------------------------------------------------------------------------------------
-constexpr int64_t kClusterAutoUnits = 96;
+// Default choice: the cluster kernel is taken while its blocks make up to about ten (sampling) or
+// three and a half (verification: two rows per position) per SM; beyond that the streaming
+// kernel's throughput wins (measured at V = 128256 and 32000).
+constexpr int64_t kClusterAutoBlocksSample = 1536, kClusterAutoBlocksVerify = 512;
 constexpr size_t kClusterSmemBytes = 200 * 1024;  // dynamic shared memory a block of the cluster kernel may use
 
 // Tiles per block that fit (roles = rows raced together: 1, or 2 for a draft/target pair).
@@ -401,16 +404,34 @@ static bool cluster_applies(const Params& p, int dt) {
   return p.c_sample == 1 && p.aligned_t && (roles == 1 || p.aligned_d) && p.rows <= 65535 && p.B <= 65535;
 }
 
-template <int DT>
-static int launch_cluster_dt(const Params& p, cudaStream_t st) {
-  auto kernel = b256::ersd_cluster_kernel<DT>;
+// Blocks per cluster: the smallest power of two that leaves a block about kClusterGroups tiles.
+static int cluster_size(const Params& p, int* out) {
   int lim = 8;
   const int ls = cluster_limit(&lim);
   if (ls != ERSD_OK) return ls;
-  // smallest power of two that lets a thread hold its share of the row in registers at once
   const int ntiles = (p.V + b256::kTile - 1) / b256::kTile;
   int CL = 1;
   while (CL < lim && CL * b256::kClusterGroups < ntiles) CL *= 2;
+  *out = CL;
+  return ERSD_OK;
+}
+
+// Whether a call that leaves the choice to the library takes the cluster kernel.
+static bool cluster_by_default(const ersd_opts& o, const Params& p, int dt) {
+  if (o.kernel_path != 0 || o.split_v != 0 || o.block_threads != 0 || !cluster_applies(p, dt)) return false;
+  int CL = 1;
+  if (cluster_size(p, &CL) != ERSD_OK) return false;
+  const int64_t blocks = (int64_t)p.B * p.rows * CL;
+  return blocks <= (p.mode == kVerify ? kClusterAutoBlocksVerify : kClusterAutoBlocksSample);
+}
+
+template <int DT>
+static int launch_cluster_dt(const Params& p, cudaStream_t st) {
+  auto kernel = b256::ersd_cluster_kernel<DT>;
+  int CL = 1;
+  const int ls = cluster_size(p, &CL);
+  if (ls != ERSD_OK) return ls;
+  const int ntiles = (p.V + b256::kTile - 1) / b256::kTile;
   const int G = (ntiles + CL - 1) / CL;  // tiles per block; they fit, see cluster_applies
   const int roles = (p.mode == kVerify && p.draft) ? 2 : 1;
   cudaLaunchConfig_t cfg;
@@ -497,8 +518,7 @@ static int verify_impl(const void* target, const void* draft, int dt, const Tree
   if (o.kernel_path > 2) return ERSD_EINVAL;
   const bool cluster_ok = chain && cmax <= 1 && cluster_applies(p, dt);
   if (o.kernel_path == 2 && !cluster_ok) return ERSD_EUNSUPPORTED;
-  if (o.kernel_path == 2 || (o.kernel_path == 0 && o.split_v == 0 && o.block_threads == 0 &&
-                             (int64_t)B * rows <= kClusterAutoUnits && cluster_ok))
+  if (cluster_ok && (o.kernel_path == 2 || cluster_by_default(o, p, dt)))
     return launch_cluster(p, dt, (cudaStream_t)stream);
   int st0 = choose_threads(o, (int64_t)B * rows, &p.threads);
   if (st0 != ERSD_OK) return st0;
@@ -563,9 +583,7 @@ int ersd_race_sample(const void* logits, ersd_dtype dt, const uint64_t* seeds, i
   p.out_key = o.out_key;
   if (o.kernel_path > 2) return ERSD_EINVAL;
   if (o.kernel_path == 2 && !cluster_applies(p, dt)) return ERSD_EUNSUPPORTED;
-  if (o.kernel_path == 2 || (o.kernel_path == 0 && o.split_v == 0 && o.block_threads == 0 &&
-                             (int64_t)B * R <= kClusterAutoUnits && cluster_applies(p, dt)))
-    return launch_cluster(p, dt, (cudaStream_t)cuda_stream);
+  if (o.kernel_path == 2 || cluster_by_default(o, p, dt)) return launch_cluster(p, dt, (cudaStream_t)cuda_stream);
   st = choose_threads(o, (int64_t)B * R, &p.threads);
   if (st != ERSD_OK) return st;
   set_chunks(p, choose_split(o, (int64_t)B * R, V, c, p.threads));
