@@ -510,14 +510,14 @@ static int verify_impl(const void* target, const void* draft, int dt, const Tree
   p.out_draft_key = o.out_draft_key;
   p.out_target_tok = o.out_target_tok;
   p.out_target_key = o.out_target_key;
-  void* ws = nullptr;
-  const int st = get_workspace(o, workspace_bytes(B, rows), &ws);
-  if (st != ERSD_OK) return st;
-  p.slots = (Slot*)ws;
   // sequences of few rows: one cluster per position (chains only: one arrival per race)
   if (o.kernel_path > 2) return ERSD_EINVAL;
   const bool cluster_ok = chain && cmax <= 1 && cluster_applies(p, dt);
   if (o.kernel_path == 2 && !cluster_ok) return ERSD_EUNSUPPORTED;
+  void* ws = nullptr;
+  const int st = get_workspace(o, workspace_bytes(B, rows), &ws);
+  if (st != ERSD_OK) return st;
+  p.slots = (Slot*)ws;
   if (cluster_ok && (o.kernel_path == 2 || cluster_by_default(o, p, dt)))
     return launch_cluster(p, dt, (cudaStream_t)stream);
   int st0 = choose_threads(o, (int64_t)B * rows, &p.threads);
@@ -741,6 +741,6 @@ const char* ersd_status_string(int status) {
 
 int ersd_last_cuda_error(void) { return g_last_cuda_error; }
 
-int ersd_version(void) { return 104; }
+int ersd_version(void) { return 105; }
 
 }  // extern "C"

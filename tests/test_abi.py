@@ -108,6 +108,17 @@ def test_argument_errors_are_found_on_the_host(L):
     o.struct_size = C.sizeof(ErsdOpts)
     o.ld_target = 4                                                          # stride below V
     assert v(p, p, 1, p, 1, 2, 8, 1.0, p, p, C.byref(o), None) == EINVAL
+    o = ErsdOpts()
+    o.struct_size = C.sizeof(ErsdOpts)
+    o.kernel_path = 3                                                        # 0, 1, 2 are the choices
+    assert v(p, p, 1, p, 1, 2, 8, 1.0, p, p, C.byref(o), None) == EINVAL
+    assert f(p, 1, p, 1, 1, 8, 1.0, p, C.byref(o), None) == EINVAL
+    o.kernel_path = 2                                                        # the cluster kernel where it cannot run
+    assert v(p, p, 1, p, 1, 32, 8, 1.0, p, p, C.byref(o), None) == EUNSUP    # more than 32 positions
+    assert v(p, C.c_void_p(0x1002), 1, p, 1, 2, 8, 1.0, p, p, C.byref(o), None) == EUNSUP  # draft rows not 16-byte aligned
+    assert t(p, p, 1, good, p, 1, 2, 8, 1.0, p, p, C.byref(o), None) == EUNSUP  # two arrivals per race
+    o.top_c = 2
+    assert f(p, 1, p, 1, 1, 8, 1.0, p, C.byref(o), None) == EUNSUP
     assert L.ersd_verify_tokens(p, None, 1, p, 1, 2, 8, 1.0, p, p, None, None) == EINVAL      # k > 0 needs tokens
     assert L.ersd_verify_tokens(p, C.c_void_p(4098), 1, p, 1, 2, 8, 1.0, p, p, None, None) == -2  # misaligned int32
     assert L.ersd_row_keys(None, 1, 8, 1.0, 0, 0, 0, 0, p, None) == EINVAL
