@@ -51,6 +51,9 @@ def main():
     ap.add_argument("--k", type=int, default=5, help="drafted positions per sequence (verification)")
     ap.add_argument("--batches", default="1,2,4,8,16,32")
     ap.add_argument("--sets", type=int, default=6, help="distinct inputs rotated between calls")
+    ap.add_argument("--plain", type=int, default=0,
+                    help="issue this many plain calls per case instead of replaying a graph and print no "
+                         "times (for a profiler's launch list)")
     args = ap.parse_args()
     binding.lib()
     if not torch.cuda.is_available():
@@ -81,6 +84,11 @@ def main():
                 binding.ersd_verify(t, d, seeds, 1.0, tok, acc, opts, st)
 
             for entry, fn, rows in (("ersd_race_sample", sample, B), ("ersd_verify", verify, B * (2 * k + 1))):
+                if args.plain:
+                    for i in range(args.plain):
+                        fn(i, torch.cuda.current_stream())
+                    torch.cuda.synchronize()
+                    continue
                 us = graph_time_us(fn)
                 print(json.dumps({"entry": entry, "B": B, "k": None if fn is sample else k, "V": V, "dtype": "bf16",
                                   "kernel": name, "us_per_call": round(us, 2), "logit_rows_per_call": rows,
