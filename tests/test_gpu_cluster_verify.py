@@ -107,6 +107,17 @@ def test_special_values_greedy_and_invalid_temperatures(ersd):
         assert same(out1, run(ersd, inp1, STREAMING))
 
 
+def test_sequence_ids_position_offsets_and_per_sequence_temperatures(ersd):
+    w = wl.Workload("opts", B=4, k=3, V=3000, dtype="bf16", sigma=0.8, T=1.0, config_id=44)
+    inp = wl.make_inputs(w)
+    inp["temps"] = torch.tensor([[0.5, 0.7, 1.0, 1.3], [1.0, 1.0, 0.0, 1.0], [2.0, 0.6, 0.6, 0.6], [1.0, 0.9, 1.0, 1.0]])
+    seq = torch.tensor([7, 7, 9, 1000000], dtype=torch.int32)
+    off = torch.tensor([0, 4, 123456, 1], dtype=torch.int32)
+    out = run(ersd, inp, CLUSTER, seq_ids=seq.cuda(), pos_offsets=off.cuda())
+    check_verify(inp, out, seq_ids=seq.numpy().astype(np.uint32), pos_offsets=off.numpy().astype(np.uint32))
+    assert same(out, run(ersd, inp, STREAMING, seq_ids=seq.cuda(), pos_offsets=off.cuda()))
+
+
 def test_identical_rows_accept_everything_and_k0(ersd):
     B, k, V = 3, 6, 40000
     g = torch.Generator().manual_seed(2)
