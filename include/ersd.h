@@ -83,7 +83,8 @@ typedef enum {
 typedef struct ersd_opts {
   uint32_t struct_size;
   uint32_t top_c;          /* ersd_race_sample: arrivals per row, 0 or 1 = winner only */
-  uint32_t split_v;        /* thread blocks per row; 0 = chosen by the library */
+  uint32_t split_v;        /* thread blocks per row (cluster kernel: per cluster, a power of two up to 16);
+                              0 = chosen by the library */
   uint32_t block_threads;  /* threads per block of the race kernel: 128, 256, or 0 = chosen by the library */
   int64_t ld_target;       /* row stride in elements of target_logits / logits; 0 = V */
   int64_t ld_draft;        /* row stride in elements of draft_logits; 0 = V */

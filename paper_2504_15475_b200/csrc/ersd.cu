@@ -336,10 +336,10 @@ static int launch(const Params& p, const TreeDesc& tree, int dt, cudaStream_t st
 // ---------------------------------------------------------------------------------------------
 // Latency path of calls of few rows: one cluster of thread blocks per position (ersd_cluster.inc).
 // ---------------------------------------------------------------------------------------------
-// Default choice: the cluster kernel is taken while its blocks make up to about ten (sampling) or
-// three and a half (verification: two rows per position) per SM; beyond that the streaming
-// kernel's throughput wins (measured at V = 128256 and 32000).
-constexpr int64_t kClusterAutoBlocksSample = 1536, kClusterAutoBlocksVerify = 512;
+// Default choice: the cluster kernel is taken while its blocks number up to 1280 (sampling: 160
+// rows of 128256 logits) or 768 (verification: two rows per position; 96 positions); beyond that
+// the streaming kernel's throughput wins (measured at V = 128256 and 32000).
+constexpr int64_t kClusterAutoBlocksSample = 1280, kClusterAutoBlocksVerify = 768;
 constexpr size_t kClusterSmemBytes = 200 * 1024;  // dynamic shared memory a block of the cluster kernel may use
 
 // Tiles per block that fit (roles = rows raced together: 1, or 2 for a draft/target pair).
@@ -404,14 +404,29 @@ static bool cluster_applies(const Params& p, int dt) {
   return p.c_sample == 1 && p.aligned_t && (roles == 1 || p.aligned_d) && p.rows <= 65535 && p.B <= 65535;
 }
 
-// Blocks per cluster: the smallest power of two that leaves a block about kClusterGroups tiles.
-static int cluster_size(const Params& p, int* out) {
+// Blocks per cluster.  Few positions: the smallest power of two that leaves a block about
+// kClusterGroups tiles (shortest path through one position).  Once such clusters would make more
+// than two blocks per SM: blocks of about twice as many tiles (measured at V = 128256: clusters
+// of 8 beat clusters of 16 from about 20 positions on, clusters of 4 never beat clusters of 8).
+static int cluster_size(const ersd_opts& o, const Params& p, int dt, int* out) {
   int lim = 8;
   const int ls = cluster_limit(&lim);
   if (ls != ERSD_OK) return ls;
   const int ntiles = (p.V + b256::kTile - 1) / b256::kTile;
+  const int roles = (p.mode == kVerify && p.draft) ? 2 : 1;
+  const int max_tiles = cluster_max_tiles(dt, roles);
+  if (o.split_v) {  // the caller's choice: a power of two that the device takes and whose blocks can stage their share
+    const int CL = (int)o.split_v;
+    if (CL > lim || (CL & (CL - 1)) != 0 || (ntiles + CL - 1) / CL > max_tiles) return ERSD_EUNSUPPORTED;
+    *out = CL;
+    return ERSD_OK;
+  }
   int CL = 1;
   while (CL < lim && CL * b256::kClusterGroups < ntiles) CL *= 2;
+  const int64_t units = (int64_t)p.B * p.rows;
+  if (units * CL > 2 * 148 && CL > 1 && (CL / 2) * 2 * b256::kClusterGroups >= ntiles &&
+      (ntiles + CL / 2 - 1) / (CL / 2) <= max_tiles)
+    CL /= 2;
   *out = CL;
   return ERSD_OK;
 }
@@ -420,16 +435,16 @@ static int cluster_size(const Params& p, int* out) {
 static bool cluster_by_default(const ersd_opts& o, const Params& p, int dt) {
   if (o.kernel_path != 0 || o.split_v != 0 || o.block_threads != 0 || !cluster_applies(p, dt)) return false;
   int CL = 1;
-  if (cluster_size(p, &CL) != ERSD_OK) return false;
+  if (cluster_size(o, p, dt, &CL) != ERSD_OK) return false;
   const int64_t blocks = (int64_t)p.B * p.rows * CL;
   return blocks <= (p.mode == kVerify ? kClusterAutoBlocksVerify : kClusterAutoBlocksSample);
 }
 
 template <int DT>
-static int launch_cluster_dt(const Params& p, cudaStream_t st) {
+static int launch_cluster_dt(const ersd_opts& o, const Params& p, cudaStream_t st) {
   auto kernel = b256::ersd_cluster_kernel<DT>;
   int CL = 1;
-  const int ls = cluster_size(p, &CL);
+  const int ls = cluster_size(o, p, DT, &CL);
   if (ls != ERSD_OK) return ls;
   const int ntiles = (p.V + b256::kTile - 1) / b256::kTile;
   const int G = (ntiles + CL - 1) / CL;  // tiles per block; they fit, see cluster_applies
@@ -451,8 +466,8 @@ static int launch_cluster_dt(const Params& p, cudaStream_t st) {
   return e == cudaSuccess ? ERSD_OK : cuda_fail(e);
 }
 
-static int launch_cluster(const Params& p, int dt, cudaStream_t st) {
-  return dt == ERSD_BF16 ? launch_cluster_dt<ERSD_BF16>(p, st) : launch_cluster_dt<ERSD_F32>(p, st);
+static int launch_cluster(const ersd_opts& o, const Params& p, int dt, cudaStream_t st) {
+  return dt == ERSD_BF16 ? launch_cluster_dt<ERSD_BF16>(o, p, st) : launch_cluster_dt<ERSD_F32>(o, p, st);
 }
 
 static int check_common(const void* logits, int dt, const uint64_t* seeds, int B, int rows, int V,
@@ -519,7 +534,7 @@ static int verify_impl(const void* target, const void* draft, int dt, const Tree
   if (st != ERSD_OK) return st;
   p.slots = (Slot*)ws;
   if (cluster_ok && (o.kernel_path == 2 || cluster_by_default(o, p, dt)))
-    return launch_cluster(p, dt, (cudaStream_t)stream);
+    return launch_cluster(o, p, dt, (cudaStream_t)stream);
   int st0 = choose_threads(o, (int64_t)B * rows, &p.threads);
   if (st0 != ERSD_OK) return st0;
   set_chunks(p, choose_split(o, (int64_t)B * rows, V, cmax, p.threads));
@@ -583,7 +598,7 @@ int ersd_race_sample(const void* logits, ersd_dtype dt, const uint64_t* seeds, i
   p.out_key = o.out_key;
   if (o.kernel_path > 2) return ERSD_EINVAL;
   if (o.kernel_path == 2 && !cluster_applies(p, dt)) return ERSD_EUNSUPPORTED;
-  if (o.kernel_path == 2 || cluster_by_default(o, p, dt)) return launch_cluster(p, dt, (cudaStream_t)cuda_stream);
+  if (o.kernel_path == 2 || cluster_by_default(o, p, dt)) return launch_cluster(o, p, dt, (cudaStream_t)cuda_stream);
   st = choose_threads(o, (int64_t)B * R, &p.threads);
   if (st != ERSD_OK) return st;
   set_chunks(p, choose_split(o, (int64_t)B * R, V, c, p.threads));

@@ -51,6 +51,7 @@ def main():
     ap.add_argument("--k", type=int, default=5, help="drafted positions per sequence (verification)")
     ap.add_argument("--batches", default="1,2,4,8,16,32")
     ap.add_argument("--sets", type=int, default=6, help="distinct inputs rotated between calls")
+    ap.add_argument("--split", type=int, default=0, help="thread blocks per row / per cluster (0: library default)")
     ap.add_argument("--plain", type=int, default=0,
                     help="issue this many plain calls per case instead of replaying a graph and print no "
                          "times (for a profiler's launch list)")
@@ -74,7 +75,7 @@ def main():
         acc = torch.empty(B, dtype=torch.int32, device="cuda")
         rows1 = [s[1][:, :1].contiguous() for s in sets]          # one draft row per sequence
         for name, path in PATHS.items():
-            opts = binding.make_opts(workspace=ws, kernel_path=path)
+            opts = binding.make_opts(workspace=ws, kernel_path=path, split_v=args.split if path else 0)
 
             def sample(i, st):
                 binding.ersd_race_sample(rows1[i % len(sets)], seeds, 1.0, tok1, opts, st)
@@ -91,7 +92,7 @@ def main():
                     continue
                 us = graph_time_us(fn)
                 print(json.dumps({"entry": entry, "B": B, "k": None if fn is sample else k, "V": V, "dtype": "bf16",
-                                  "kernel": name, "us_per_call": round(us, 2), "logit_rows_per_call": rows,
+                                  "kernel": name, "split": args.split if path else 0, "us_per_call": round(us, 2), "logit_rows_per_call": rows,
                                   "timing": "CUDA graph replay, 30 calls per graph"}), flush=True)
 
 

@@ -235,3 +235,24 @@ def test_screening_keys_too_close_to_call_are_decided_exactly(ersd, gap):
     assert tok[:, 0, 0].cpu().tolist() == want
     tok_s, key_s = sample(ersd, logits, seeds, T, STREAMING)
     assert (tok == tok_s).all() and (key == key_s).all()
+
+
+def test_every_cluster_size_gives_the_same_result(ersd):
+    B, V = 5, 40000                                   # 20 tiles: clusters of 1 to 16 blocks stage 20 to 2 tiles each
+    g = torch.Generator().manual_seed(77)
+    logits = wl.zipf_rows(B, V, g, "cpu").view(B, 1, V).to(torch.bfloat16)
+    seeds = wl.make_seeds(12, 0, B)
+    ref_tok, ref_key = sample(ersd, logits, seeds, 1.0, STREAMING)
+    assert check_sample(logits, seeds, 1.0, ref_tok, ref_key) == 0
+    for blocks in (1, 2, 4, 8, 16):
+        tok, key = sample(ersd, logits, seeds, 1.0, CLUSTER, split_v=blocks)
+        assert (tok == ref_tok).all() and (key == ref_key).all()
+    tok = torch.empty(B, 1, 1, dtype=torch.int32, device="cuda")
+    for bad in (3, 32):                               # not a power of two; more than a cluster holds
+        with pytest.raises(ersd.ErsdError) as e:
+            ersd.ersd_race_sample(logits.cuda(), seeds.cuda(), 1.0, tok, ersd.make_opts(kernel_path=CLUSTER, split_v=bad))
+        assert e.value.status == -3
+    big = torch.zeros(1, 1, 300000, dtype=torch.float32).cuda()   # 147 tiles of fp32: too many for one block
+    with pytest.raises(ersd.ErsdError) as e:
+        ersd.ersd_race_sample(big, seeds[:1].cuda(), 1.0, tok[:1], ersd.make_opts(kernel_path=CLUSTER, split_v=1))
+    assert e.value.status == -3
