@@ -14,7 +14,7 @@ from typing import Optional, Sequence
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libersd.so")
+LIB_PATH = os.environ.get("ERSD_LIBRARY") or os.path.join(_HERE, "libersd.so")  # ERSD_LIBRARY: another build of libersd
 
 ERSD_F32, ERSD_BF16 = 0, 1
 ERSD_OK = 0

@@ -756,6 +756,6 @@ const char* ersd_status_string(int status) {
 
 int ersd_last_cuda_error(void) { return g_last_cuda_error; }
 
-int ersd_version(void) { return 105; }
+int ersd_version(void) { return 106; }
 
 }  // extern "C"
