@@ -398,6 +398,25 @@ def test_race_sample_first_arrivals(ersd, c, split):
     check_sample(logits, seeds, 0.9, tok, key, c=c)
 
 
+@pytest.mark.parametrize("threads", [128, 256])
+@pytest.mark.parametrize("c,split", [(2, 1), (8, 0), (8, 7), (32, 2), (32, 16)])
+def test_many_arrivals_at_full_vocabulary(ersd, c, split, threads):
+    """Batch drafting's first c arrivals over 128256 tokens: chunks of many tiles, thresholds that
+    start from the block-wide c-th smallest screening key, survivors decided several at a time."""
+    B, R, V = 2, 2, 128256
+    g = torch.Generator().manual_seed(100 * c + split)
+    logits = wl.zipf_rows(B * R, V, g, "cpu").view(B, R, V).to(torch.bfloat16)
+    logits[1, 1, 7::2] = float("-inf")               # half of one row masked
+    seeds = wl.make_seeds(17, c, B)
+    tok = torch.empty(B, R, c, dtype=torch.int32, device="cuda")
+    key = torch.empty(B, R, c, dtype=torch.float32, device="cuda")
+    ersd.ersd_race_sample(logits.cuda(), seeds.cuda(), 0.8, tok,
+                          ersd.make_opts(top_c=c, split_v=split, block_threads=threads, out_key=key))
+    torch.cuda.synchronize()
+    assert check_sample(logits, seeds, 0.8, tok, key, c=c) == 0
+    assert all(len(set(r.tolist())) == c for r in tok.view(-1, c).cpu())
+
+
 def test_race_sample_draft_then_verify_is_consistent(ersd):
     """Drafting with race_sample and verifying with ersd_verify see the same draft winners."""
     w = wl.scaled(wl.CONFIGS["c2"], B=4)
