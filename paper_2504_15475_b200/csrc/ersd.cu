@@ -92,12 +92,25 @@ struct Params {
 // ---------------------------------------------------------------------------------------------
 namespace b256 {
 constexpr int kThreads = 256, kMinBlocks = 4;
+constexpr bool kMany = false;
 #include "ersd_kernel.inc"
 }  // namespace b256
 namespace b128 {
 constexpr int kThreads = 128, kMinBlocks = 8;
+constexpr bool kMany = false;
 #include "ersd_kernel.inc"
 }  // namespace b128
+// The same two for calls with races that want several arrivals (tree and batch drafting, top_c > 1).
+namespace b256m {
+constexpr int kThreads = 256, kMinBlocks = 4;
+constexpr bool kMany = true;
+#include "ersd_kernel.inc"
+}  // namespace b256m
+namespace b128m {
+constexpr int kThreads = 128, kMinBlocks = 8;
+constexpr bool kMany = true;
+#include "ersd_kernel.inc"
+}  // namespace b128m
 namespace b256 {
 #include "ersd_cluster.inc"
 }  // namespace b256
@@ -295,11 +308,15 @@ static int prefer_shared_memory() {
   std::lock_guard<std::mutex> lock(m);
   if (!done[dev]) {
     e = cudaSuccess;
-    const void* kernels[4] = {(const void*)b256::ersd_race_kernel<ERSD_BF16>, (const void*)b256::ersd_race_kernel<ERSD_F32>,
-                              (const void*)b128::ersd_race_kernel<ERSD_BF16>, (const void*)b128::ersd_race_kernel<ERSD_F32>};
-    const int smem[4] = {(int)sizeof(b256::Shared<ERSD_BF16>), (int)sizeof(b256::Shared<ERSD_F32>),
-                         (int)sizeof(b128::Shared<ERSD_BF16>), (int)sizeof(b128::Shared<ERSD_F32>)};
-    for (int q = 0; q < 4 && e == cudaSuccess; ++q) {
+    const void* kernels[8] = {(const void*)b256::ersd_race_kernel<ERSD_BF16>, (const void*)b256::ersd_race_kernel<ERSD_F32>,
+                              (const void*)b128::ersd_race_kernel<ERSD_BF16>, (const void*)b128::ersd_race_kernel<ERSD_F32>,
+                              (const void*)b256m::ersd_race_kernel<ERSD_BF16>, (const void*)b256m::ersd_race_kernel<ERSD_F32>,
+                              (const void*)b128m::ersd_race_kernel<ERSD_BF16>, (const void*)b128m::ersd_race_kernel<ERSD_F32>};
+    const int smem[8] = {(int)sizeof(b256::Shared<ERSD_BF16>), (int)sizeof(b256::Shared<ERSD_F32>),
+                         (int)sizeof(b128::Shared<ERSD_BF16>), (int)sizeof(b128::Shared<ERSD_F32>),
+                         (int)sizeof(b256m::Shared<ERSD_BF16>), (int)sizeof(b256m::Shared<ERSD_F32>),
+                         (int)sizeof(b128m::Shared<ERSD_BF16>), (int)sizeof(b128m::Shared<ERSD_F32>)};
+    for (int q = 0; q < 8 && e == cudaSuccess; ++q) {
       e = cudaFuncSetAttribute(kernels[q], cudaFuncAttributePreferredSharedMemoryCarveout,
                                cudaSharedmemCarveoutMaxShared);
       if (e == cudaSuccess)
@@ -311,14 +328,31 @@ static int prefer_shared_memory() {
   return ERSD_OK;
 }
 
-static int launch(const Params& p, const TreeDesc& tree, int dt, cudaStream_t st) {
+// `many`: some race of the call wants several arrivals (a tree node with several children,
+// top_c > 1).  Calls of up to two rows per SM then take the variant of the kernel that pools the
+// block's decided indices (measured: a star of 8 at B=1 48 -> 42 us, the 17-node tree 35 -> 33 us;
+// at 544 rows the pooling costs 0.7 % instead).
+static int launch(const Params& p, const TreeDesc& tree, int dt, bool many, cudaStream_t st) {
+  many = many && (int64_t)p.B * p.rows <= 2 * 148;
   // grid (sequence, row in launch order, chunk): blocks are dispatched x fastest, z slowest, which
   // is the chunk-major order the kernel counts on, and the kernel needs no division to decode
   if (p.rows > 65535 || p.S > 65535) return ERSD_EUNSUPPORTED;
   const dim3 grid((unsigned)p.B, (unsigned)p.rows, (unsigned)p.S);
   const int pst = prefer_shared_memory();
   if (pst != ERSD_OK) return pst;
-  if (p.threads == 128) {
+  if (many) {
+    if (p.threads == 128) {
+      if (dt == ERSD_BF16)
+        b128m::ersd_race_kernel<ERSD_BF16><<<grid, 128, sizeof(b128m::Shared<ERSD_BF16>), st>>>(p, tree);
+      else
+        b128m::ersd_race_kernel<ERSD_F32><<<grid, 128, sizeof(b128m::Shared<ERSD_F32>), st>>>(p, tree);
+    } else {
+      if (dt == ERSD_BF16)
+        b256m::ersd_race_kernel<ERSD_BF16><<<grid, 256, sizeof(b256m::Shared<ERSD_BF16>), st>>>(p, tree);
+      else
+        b256m::ersd_race_kernel<ERSD_F32><<<grid, 256, sizeof(b256m::Shared<ERSD_F32>), st>>>(p, tree);
+    }
+  } else if (p.threads == 128) {
     if (dt == ERSD_BF16)
       b128::ersd_race_kernel<ERSD_BF16><<<grid, 128, sizeof(b128::Shared<ERSD_BF16>), st>>>(p, tree);
     else
@@ -538,7 +572,7 @@ static int verify_impl(const void* target, const void* draft, int dt, const Tree
   int st0 = choose_threads(o, (int64_t)B * rows, &p.threads);
   if (st0 != ERSD_OK) return st0;
   set_chunks(p, choose_split(o, (int64_t)B * rows, V, cmax, p.threads));
-  return launch(p, tree, dt, (cudaStream_t)stream);
+  return launch(p, tree, dt, cmax > 1, (cudaStream_t)stream);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -610,7 +644,7 @@ int ersd_race_sample(const void* logits, ersd_dtype dt, const uint64_t* seeds, i
   }
   TreeDesc tree;
   memset(&tree, 0, sizeof tree);
-  return launch(p, tree, dt, (cudaStream_t)cuda_stream);
+  return launch(p, tree, dt, c > 1, (cudaStream_t)cuda_stream);
 }
 
 int ersd_verify(const void* target_logits, const void* draft_logits, ersd_dtype dt,
@@ -756,6 +790,6 @@ const char* ersd_status_string(int status) {
 
 int ersd_last_cuda_error(void) { return g_last_cuda_error; }
 
-int ersd_version(void) { return 106; }
+int ersd_version(void) { return 107; }
 
 }  // extern "C"
