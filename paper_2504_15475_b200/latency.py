@@ -45,6 +45,37 @@ def graph_time_us(call, calls_per_graph=30, replays=20):
     return e0.elapsed_time(e1) * 1e3 / (calls_per_graph * replays)
 
 
+def time_trees(args):
+    """ersd_verify_tree on the draft-tree shapes of the workloads module."""
+    V = args.V
+    shapes = (("root with 4 children, chains to depth 4", wl.TREE_4x4), ("SpecInfer shape", wl.TREE_SPECINFER),
+              ("star of 8", wl.star_parent(8)), ("chain of 16", wl.chain_parent(16)))
+    for name, parent in shapes:
+        n = len(parent)
+        for B in [int(x) for x in args.batches.split(",")]:
+            gen = torch.Generator().manual_seed(2000 + B)
+            sets = []
+            for _ in range(min(args.sets, 4)):
+                t = wl.zipf_rows(B * n, V, gen, "cpu").view(B, n, V)
+                d = t + torch.randn(B, n, V, generator=gen)
+                sets.append((t.to(torch.bfloat16).cuda(), d.to(torch.bfloat16).cuda()))
+            seeds = wl.make_seeds(78, B, B).cuda()
+            D = binding.ersd_tree_depth(parent)
+            tok = torch.empty(B, D + 1, dtype=torch.int32, device="cuda")
+            acc = torch.empty(B, dtype=torch.int32, device="cuda")
+            ws = torch.zeros(binding.ersd_workspace_bytes(B, n), dtype=torch.uint8, device="cuda")
+            binding.ersd_workspace_init(ws)
+            opts = binding.make_opts(workspace=ws, split_v=args.split)
+
+            def call(i, st):
+                t, d = sets[i % len(sets)]
+                binding.ersd_verify_tree(t, d, parent, seeds, 1.0, tok, acc, opts, st)
+
+            print(json.dumps({"entry": "ersd_verify_tree", "tree": name, "nodes": n, "B": B, "V": V, "dtype": "bf16",
+                              "us_per_call": round(graph_time_us(call), 2),
+                              "timing": "CUDA graph replay, 30 calls per graph"}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--V", type=int, default=128256)
@@ -52,6 +83,8 @@ def main():
     ap.add_argument("--batches", default="1,2,4,8,16,32")
     ap.add_argument("--sets", type=int, default=6, help="distinct inputs rotated between calls")
     ap.add_argument("--split", type=int, default=0, help="thread blocks per row / per cluster (0: library default)")
+    ap.add_argument("--trees", action="store_true",
+                    help="time ersd_verify_tree on draft trees (streaming kernel) instead of the two entries above")
     ap.add_argument("--plain", type=int, default=0,
                     help="issue this many plain calls per case instead of replaying a graph and print no "
                          "times (for a profiler's launch list)")
@@ -60,6 +93,9 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("needs a CUDA device")
     V, k = args.V, args.k
+    if args.trees:
+        time_trees(args)
+        return
     for B in [int(x) for x in args.batches.split(",")]:
         gen = torch.Generator().manual_seed(1000 + B)
         sets = []
