@@ -1,0 +1,100 @@
+"""Differential test of the two kernels: seeded random shapes, temperatures and masks; the cluster
+kernel and the streaming kernel must agree bit for bit (tokens, accept lengths, per-row winners
+and keys), and a sample of the cases is also checked against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2504_15475_b200 import workloads as wl
+
+from parity_util import check_verify
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ersd():
+    from paper_2504_15475_b200 import binding
+    binding.lib()
+    assert torch.cuda.is_available()
+    return binding
+
+
+def random_case(rng: np.random.Generator, g: torch.Generator):
+    B = int(rng.integers(1, 6))
+    k = int(rng.integers(0, 9))
+    V = int(rng.choice([int(rng.integers(1, 64)), int(rng.integers(64, 5000)), int(rng.integers(5000, 70000)),
+                        int(rng.integers(70000, 160000))]))
+    V8 = (V + 7) // 8 * 8                       # rows padded to 16-byte boundaries
+    dtype = "bf16" if rng.random() < 0.7 else "f32"
+    T = float(rng.choice([0.0, 0.3, 0.7, 1.0, 1.0, 1.7]))
+    style = rng.integers(0, 4)
+    if style == 0:
+        t = wl.zipf_rows(B * (k + 1), V, g, "cpu").view(B, k + 1, V)
+    elif style == 1:
+        t = torch.randn(B, k + 1, V, generator=g) * float(rng.uniform(0.1, 4.0))
+    elif style == 2:                            # few distinct values: many ties in bf16
+        t = torch.randint(-3, 4, (B, k + 1, V), generator=g).float() * 0.5
+    else:                                       # peaked
+        t = torch.full((B, k + 1, V), -20.0) + torch.randn(B, k + 1, V, generator=g)
+        t[..., int(rng.integers(0, V))] = 3.0
+    d = t[:, :k] + float(rng.uniform(0.0, 1.5)) * torch.randn(B, k, V, generator=g)
+    if rng.random() < 0.4:                      # masked ranges, infinities, NaNs
+        lo = int(rng.integers(0, V))
+        t[:, :, lo:lo + int(rng.integers(1, V + 1))] = float("-inf")
+        if k > 0 and rng.random() < 0.5:
+            d[:, 0, int(rng.integers(0, V))] = float("inf")
+        if rng.random() < 0.3:
+            t[0, 0, int(rng.integers(0, V))] = float("nan")
+    big_t = torch.full((B, k + 1, V8), 70.0)
+    big_d = torch.full((B, max(k, 1), V8), 70.0)
+    big_t[:, :, :V] = t
+    if k > 0:
+        big_d[:, :k, :V] = d
+    temps = None
+    if rng.random() < 0.3:
+        temps = torch.tensor(rng.choice([0.0, 0.5, 1.0, 2.0], size=(B, k + 1)), dtype=torch.float32)
+    return dict(B=B, k=k, V=V, ld=V8, dtype=dtype, T=T, temps=temps,
+                target=wl._storage(big_t, dtype), draft=wl._storage(big_d[:, :k].contiguous(), dtype) if k > 0 else None,
+                seeds=wl.make_seeds(int(rng.integers(0, 1 << 30)), 0, B))
+
+
+def run(ersd, case, path):
+    B, k, V, ld = case["B"], case["k"], case["V"], case["ld"]
+    out = dict(tokens=torch.full((B, k + 1), -7, dtype=torch.int32, device="cuda"),
+               accept_len=torch.full((B,), -7, dtype=torch.int32, device="cuda"),
+               target_tok=torch.full((B, k + 1), -7, dtype=torch.int32, device="cuda"),
+               target_key=torch.full((B, k + 1), -7.0, dtype=torch.float32, device="cuda"),
+               draft_tok=torch.full((B, k), -7, dtype=torch.int32, device="cuda"),
+               draft_key=torch.full((B, k), -7.0, dtype=torch.float32, device="cuda"))
+    kw = dict(ld_target=ld, ld_draft=ld, kernel_path=path, out_target_tok=out["target_tok"],
+              out_target_key=out["target_key"])
+    if k > 0:
+        kw.update(out_draft_tok=out["draft_tok"], out_draft_key=out["draft_key"])
+    if case["temps"] is not None:
+        tp = case["temps"].cuda()
+        kw.update(temps=tp, temp_strides=(tp.stride(0), tp.stride(1)))
+    ersd.ersd_verify(case["target"].cuda(), case["draft"].cuda() if k > 0 else None, case["seeds"].cuda(), case["T"],
+                     out["tokens"], out["accept_len"], ersd.make_opts(**kw), V=V)
+    torch.cuda.synchronize()
+    return out
+
+
+@pytest.mark.parametrize("chunk", range(6))
+def test_random_cases_agree_between_the_kernels(ersd, chunk):
+    rng = np.random.default_rng(1234 + chunk)
+    g = torch.Generator().manual_seed(99 + chunk)
+    for n in range(25):
+        case = random_case(rng, g)
+        a = run(ersd, case, 2)
+        b = run(ersd, case, 1)
+        for name in a:
+            same = (a[name] == b[name]) | (torch.isnan(a[name].float()) & torch.isnan(b[name].float()))
+            assert same.all(), (chunk, n, name, {q: case[q] for q in ("B", "k", "V", "dtype", "T")}, a[name], b[name])
+        if n % 5 == 0 and case["temps"] is None:       # and the oracle agrees with both
+            V = case["V"]
+            inp = dict(target=case["target"][:, :, :V].contiguous(),
+                       draft=case["draft"][:, :, :V].contiguous() if case["k"] > 0 else
+                       torch.empty(case["B"], 0, V, dtype=case["target"].dtype),
+                       seeds=case["seeds"], T=case["T"], temps=None, parent=None)
+            check_verify(inp, a)
