@@ -1,6 +1,8 @@
 """Differential test of the two kernels: seeded random shapes, temperatures and masks; the cluster
 kernel and the streaming kernel must agree bit for bit (tokens, accept lengths, per-row winners
 and keys), and a sample of the cases is also checked against the CPU oracle."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -80,7 +82,7 @@ def run(ersd, case, path):
     return out
 
 
-@pytest.mark.parametrize("chunk", range(6))
+@pytest.mark.parametrize("chunk", range(int(os.environ.get("ERSD_DIFFERENTIAL_CHUNKS", "6"))))  # 25 cases each
 def test_random_cases_agree_between_the_kernels(ersd, chunk):
     rng = np.random.default_rng(1234 + chunk)
     g = torch.Generator().manual_seed(99 + chunk)
