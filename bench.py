@@ -33,7 +33,7 @@ if ROOT not in sys.path:
 # profiles/: dram bytes (read + write) per algorithmic byte of one launch, and the library version
 # the counters were taken at
 DRAM_BYTES_PER_ALGORITHMIC_BYTE = 1.024
-TRAFFIC_AT_VERSION = 107
+TRAFFIC_AT_VERSION = 108  # (version 108 changed the cluster kernel only: the counters of version 107 stand)
 SM_COUNT = 148
 
 METRIC = "race-verified logit rows/s at V=128256 bf16 (B*(k+1) rows)"

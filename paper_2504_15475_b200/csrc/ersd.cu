@@ -393,15 +393,18 @@ static int cluster_limit(int* out) {
   if (dev < 0 || dev >= 64) return ERSD_EUNSUPPORTED;
   std::lock_guard<std::mutex> lock(m);
   if (!limit[dev]) {
-    const void* kernels[2] = {(const void*)b256::ersd_cluster_kernel<ERSD_BF16>,
-                              (const void*)b256::ersd_cluster_kernel<ERSD_F32>};
-    const int smem[2] = {(int)kClusterSmemBytes, (int)kClusterSmemBytes};
+    const void* kernels[4] = {(const void*)b256::ersd_cluster_kernel<ERSD_BF16, 1>,
+                              (const void*)b256::ersd_cluster_kernel<ERSD_F32, 1>,
+                              (const void*)b256::ersd_cluster_kernel<ERSD_BF16, 2>,
+                              (const void*)b256::ersd_cluster_kernel<ERSD_F32, 2>};
+    const int smem[4] = {(int)kClusterSmemBytes, (int)kClusterSmemBytes, (int)kClusterSmemBytes,
+                         (int)kClusterSmemBytes};
     int lim = 16;
-    for (int q = 0; q < 2; ++q) {
+    for (int q = 0; q < 4; ++q) {
       e = cudaFuncSetAttribute(kernels[q], cudaFuncAttributeMaxDynamicSharedMemorySize, smem[q]);
       if (e != cudaSuccess) return cuda_fail(e);
     }
-    for (int q = 0; q < 2 && lim == 16; ++q) {
+    for (int q = 0; q < 4 && lim == 16; ++q) {
       e = cudaFuncSetAttribute(kernels[q], cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
       int n = 0;
       if (e == cudaSuccess) {
@@ -476,13 +479,13 @@ static bool cluster_by_default(const ersd_opts& o, const Params& p, int dt) {
 
 template <int DT>
 static int launch_cluster_dt(const ersd_opts& o, const Params& p, cudaStream_t st) {
-  auto kernel = b256::ersd_cluster_kernel<DT>;
+  const int roles = (p.mode == kVerify && p.draft) ? 2 : 1;
+  auto kernel = roles == 2 ? b256::ersd_cluster_kernel<DT, 2> : b256::ersd_cluster_kernel<DT, 1>;
   int CL = 1;
   const int ls = cluster_size(o, p, DT, &CL);
   if (ls != ERSD_OK) return ls;
   const int ntiles = (p.V + b256::kTile - 1) / b256::kTile;
   const int G = (ntiles + CL - 1) / CL;  // tiles per block; they fit, see cluster_applies
-  const int roles = (p.mode == kVerify && p.draft) ? 2 : 1;
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
   cfg.gridDim = dim3((unsigned)CL, (unsigned)p.rows, (unsigned)p.B);
@@ -790,6 +793,6 @@ const char* ersd_status_string(int status) {
 
 int ersd_last_cuda_error(void) { return g_last_cuda_error; }
 
-int ersd_version(void) { return 107; }
+int ersd_version(void) { return 108; }
 
 }  // extern "C"
