@@ -102,11 +102,13 @@ typedef struct ersd_opts {
   float* out_key;          /* device, nullable, ersd_race_sample: [B, R, c] keys of the arrivals */
   void* workspace;         /* device scratch or NULL (library-owned) */
   size_t workspace_bytes;
-  uint32_t kernel_path;    /* ersd_race_sample, ersd_verify, ersd_verify_tokens, ersd_verify_noalloc:
+  uint32_t kernel_path;    /* ersd_race_sample, ersd_verify, ersd_verify_tokens, ersd_verify_noalloc, and
+                              ersd_verify_tree on a tree without branching:
                               0 = chosen by the library, 1 = the streaming kernel, 2 = the cluster kernel
                               (one thread-block cluster per position, for calls of few rows;
-                              ERSD_EUNSUPPORTED where it does not apply: top_c > 1, rows not 16-byte
-                              aligned, B or R > 65535, k + 1 > 32, or a vocabulary too long for eight
+                              ERSD_EUNSUPPORTED where it does not apply: top_c > 1, a node with several
+                              children, rows not 16-byte aligned, B or R > 65535, more than 32 rows per
+                              sequence, or a vocabulary too long for eight
                               blocks to stage in shared memory: beyond about 320 k entries in bf16,
                               160 k in fp32, halved when draft rows are raced along) */
   uint32_t reserved1;

@@ -564,7 +564,7 @@ static int verify_impl(const void* target, const void* draft, int dt, const Tree
   p.out_target_key = o.out_target_key;
   // sequences of few rows: one cluster per position (chains only: one arrival per race)
   if (o.kernel_path > 2) return ERSD_EINVAL;
-  const bool cluster_ok = chain && cmax <= 1 && cluster_applies(p, dt);
+  const bool cluster_ok = cmax <= 1 && cluster_applies(p, dt);  // (a tree without branching is the chain 0 -> 1 -> ...)
   if (o.kernel_path == 2 && !cluster_ok) return ERSD_EUNSUPPORTED;
   void* ws = nullptr;
   const int st = get_workspace(o, workspace_bytes(B, rows), &ws);

@@ -220,6 +220,25 @@ def test_screening_keys_too_close_to_call(ersd, gap):
     assert (out["target_tok"].cpu().numpy() == want).all()
 
 
+def test_a_chain_given_as_a_tree(ersd):
+    """A draft tree without branching (what the tree builder returns when first children are
+    accepted often) takes the cluster kernel too, with the tree entry point's output layout."""
+    parent, expected = ersd.ersd_optimal_tree([0.9, 0.02], 6)
+    assert list(parent) == wl.chain_parent(6) and expected > 3.0
+    w = wl.Workload("chain_tree", B=3, k=6, V=30000, dtype="bf16", sigma=0.5, T=0.9, config_id=61,
+                    parent=tuple(parent))
+    inp = wl.make_inputs(w)
+    outs = {}
+    for path in (CLUSTER, STREAMING):
+        out = ersd.verify(inp["target"].cuda(), inp["draft"].cuda(), inp["seeds"].cuda(), inp["T"],
+                          parent=list(parent), want_rows=True, kernel_path=path)
+        torch.cuda.synchronize()
+        check_verify(inp, out)
+        outs[path] = out
+    assert same(outs[CLUSTER], outs[STREAMING])
+    assert (outs[CLUSTER]["draft_tok"][:, 0] == -1).all()
+
+
 def test_where_the_cluster_kernel_does_not_apply(ersd):
     B, V = 2, 1024
     seeds = wl.make_seeds(1, 0, B).cuda()
