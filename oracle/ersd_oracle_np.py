@@ -72,7 +72,13 @@ def first_arrivals(t: np.ndarray, c: int) -> np.ndarray:
     return out
 
 
-def verify(target: np.ndarray, draft: np.ndarray, seeds, T: float):
+def _temperature(T: float, temps, b: int, r: int) -> float:
+    """Temperature of row r of sequence b: temps[b][r] where a table is given, else T.  The
+    draft row and the target row of a position are raced at the same temperature."""
+    return float(T) if temps is None else float(temps[b][r])
+
+
+def verify(target: np.ndarray, draft: np.ndarray, seeds, T: float, temps=None):
     B, rows, V = target.shape
     k = rows - 1
     tokens = np.full((B, rows), -1, dtype=np.int64)
@@ -80,11 +86,12 @@ def verify(target: np.ndarray, draft: np.ndarray, seeds, T: float):
     for b in range(B):
         L = 0
         for j in range(rows):
-            tp = first_arrivals(arrival_times(target[b, j], T, int(seeds[b]), b, j), 1)[0]
+            Tj = _temperature(T, temps, b, j)
+            tp = first_arrivals(arrival_times(target[b, j], Tj, int(seeds[b]), b, j), 1)[0]
             tokens[b, j] = tp
             if j == k:
                 break
-            tq = first_arrivals(arrival_times(draft[b, j], T, int(seeds[b]), b, j), 1)[0]
+            tq = first_arrivals(arrival_times(draft[b, j], Tj, int(seeds[b]), b, j), 1)[0]
             if tq != tp or tp < 0:
                 break
             L += 1
@@ -92,7 +99,7 @@ def verify(target: np.ndarray, draft: np.ndarray, seeds, T: float):
     return tokens, accept
 
 
-def verify_tree(target: np.ndarray, draft: np.ndarray, parent, seeds, T: float):
+def verify_tree(target: np.ndarray, draft: np.ndarray, parent, seeds, T: float, temps=None):
     B, nodes, V = target.shape
     children = [[] for _ in range(nodes)]
     for m in range(1, nodes):
@@ -101,11 +108,12 @@ def verify_tree(target: np.ndarray, draft: np.ndarray, parent, seeds, T: float):
     for b in range(B):
         y, cur = [], 0
         while True:
-            w = first_arrivals(arrival_times(target[b, cur], T, int(seeds[b]), b, cur), 1)[0]
+            Tn = _temperature(T, temps, b, cur)
+            w = first_arrivals(arrival_times(target[b, cur], Tn, int(seeds[b]), b, cur), 1)[0]
             y.append(int(w))
             nxt = None
             if children[cur] and w >= 0:
-                arr = first_arrivals(arrival_times(draft[b, cur], T, int(seeds[b]), b, cur),
+                arr = first_arrivals(arrival_times(draft[b, cur], Tn, int(seeds[b]), b, cur),
                                      len(children[cur]))
                 for r, m in enumerate(children[cur]):
                     if arr[r] == w:

@@ -243,3 +243,120 @@ def test_token_given_verification_outcomes_of_algorithm_2():
     cut = oracle.verify_tokens(tgt3, d, seeds, T=1.0)
     assert (cut["accept_len"] == 1).all() and (cut["tokens"][:, 2:] == -1).all()
     assert (cut["tokens"][:, :2] == w3[:, :2, 0]).all()
+
+
+# ----------------------------------------------------------------------------- per-row temperatures
+def distinct_temps(B, rows):
+    """A temperature table in which every entry differs (0.35 .. ~2), as float32."""
+    return (0.35 + 0.11 * np.arange(B * rows).reshape(B, rows)).astype(np.float32)
+
+
+def test_per_row_temperatures_reach_their_rows_in_sequence_verification():
+    """p = softmax(z / T) with T the temperature of THAT row (Section 3: the winner of a race is
+    a sample of the row's law); the draft row of position j is raced at the temperature of
+    target row j, with the same race variables."""
+    rng = np.random.default_rng(21)
+    B, k, V = 3, 4, 96
+    rows = k + 1
+    tgt = (3.0 * rng.normal(size=(B, rows, V))).astype(np.float32)
+    drf = (tgt + 0.3 * rng.normal(size=(B, rows, V))).astype(np.float32)[:, :k]
+    seeds = np.array([11, 22, 33], dtype=np.uint64)
+    t = distinct_temps(B, rows)
+    out = oracle.verify(tgt, drf, seeds, T=123.0, temps=t)      # the scalar must be ignored
+    differs = 0
+    for b in range(B):
+        for j in range(rows):
+            kt = oracle.row_keys(tgt[b, j], float(t[b, j]), int(seeds[b]), b, j)
+            assert out["target_tok"][b, j] == np.argmin(kt)
+            assert out["target_key"][b, j, 0] == kt.min()
+            # the same row raced at a neighbouring entry's temperature has another key
+            other = oracle.row_keys(tgt[b, j], float(t[(b + 1) % B, (j + 1) % rows]), int(seeds[b]), b, j)
+            differs += int(other.min() != kt.min())
+            if j < k:
+                kd = oracle.row_keys(drf[b, j], float(t[b, j]), int(seeds[b]), b, j)
+                assert out["draft_tok"][b, j] == np.argmin(kd)
+                assert out["draft_key"][b, j, 0] == kd.min()
+    assert differs == B * rows
+    # the separately written numpy statement, given the same table, agrees
+    tok_np, acc_np = onp.verify(tgt, drf, seeds, 123.0, temps=t.astype(np.float64))
+    assert (acc_np == out["accept_len"]).all()
+    for b in range(B):
+        L = acc_np[b]
+        assert list(tok_np[b, :L + 1]) == list(out["tokens"][b, :L + 1])
+    # and the table matters: one scalar temperature gives other winners somewhere
+    flat = oracle.verify(tgt, drf, seeds, T=1.0)
+    assert (flat["target_key"][..., 0] != out["target_key"][..., 0]).any()
+
+
+def test_per_row_temperatures_reach_their_nodes_in_tree_verification():
+    """Algorithm 5 with one temperature per node: node n's target row and draft row are both
+    raced at temps[b, n]."""
+    rng = np.random.default_rng(22)
+    parent = wl.TREE_SPECINFER
+    nodes = len(parent)
+    B, V = 2, 80
+    tgt = (3.0 * rng.normal(size=(B, nodes, V))).astype(np.float32)
+    drf = (tgt + 0.3 * rng.normal(size=(B, nodes, V))).astype(np.float32)
+    seeds = np.array([5, 6], dtype=np.uint64)
+    t = distinct_temps(B, nodes)
+    res = oracle.verify_tree(tgt, drf, parent, seeds, T=55.0, temps=t)
+    _, _, nchild, _ = oracle.tree_shape(parent)
+    for b in range(B):
+        for n in range(nodes):
+            kt = oracle.row_keys(tgt[b, n], float(t[b, n]), int(seeds[b]), b, n)
+            assert res["target_tok"][b, n] == np.argmin(kt)
+            if nchild[n]:
+                kd = oracle.row_keys(drf[b, n], float(t[b, n]), int(seeds[b]), b, n)
+                want = np.argsort(kd, kind="stable")[:nchild[n]]
+                assert list(res["arrivals"][b, n, :nchild[n]]) == list(want)
+    ys = onp.verify_tree(tgt, drf, list(parent), seeds, 55.0, temps=t.astype(np.float64))
+    for b in range(B):
+        n = res["accept_len"][b] + 1
+        assert list(res["tokens"][b, :n]) == ys[b]
+
+
+def test_winner_law_per_row_temperature():
+    """Losslessness (Section 3) row by row: in ONE call whose rows alternate between two
+    temperatures, the winners of the rows at T_a follow softmax(z / T_a) and those at T_b follow
+    softmax(z / T_b).  Negative controls: the same counts fit neither the other row's
+    temperature (indices swapped) nor the scalar T of the call."""
+    from scipy import stats
+    z = np.array([0.4, -1.1, 1.3, 0.0, 0.7], np.float32)
+    V, R = z.shape[0], 120_000
+    Ta, Tb, Tscalar = 0.5, 1.6, 1.0
+    logits = np.broadcast_to(z, (2, R, V)).copy()
+    temps = np.empty((2, R), np.float32)
+    temps[0, 0::2], temps[0, 1::2] = Ta, Tb
+    temps[1, 0::2], temps[1, 1::2] = Tb, Ta
+    tok, _ = oracle.race_sample(logits, seeds=[77, 78], T=Tscalar, temps=temps)
+    tok = tok[..., 0]
+    groups = {(0, 0): Ta, (0, 1): Tb, (1, 0): Tb, (1, 1): Ta}
+    for (b, parity), T_true in groups.items():
+        cnt = np.bincount(tok[b, parity::2], minlength=V)
+        n = cnt.sum()
+        T_other = Tb if T_true == Ta else Ta
+        assert stats.chisquare(cnt, softmax(z, T_true) * n).pvalue > 1e-3, (b, parity)
+        assert stats.chisquare(cnt, softmax(z, T_other) * n).pvalue < 1e-12
+        assert stats.chisquare(cnt, softmax(z, Tscalar) * n).pvalue < 1e-12
+
+
+def test_shared_race_at_per_row_temperature_matches_the_closed_form():
+    """Draft and target row of a position share the race AND the temperature: the match rate of
+    position j is sum_i 1 / sum_l max(p_l / p_i, q_l / q_i) with p, q = softmax(. / temps[b, j])
+    (the coupling of Section 3), not the value at another row's temperature."""
+    rng = np.random.default_rng(23)
+    k, V, B = 2, 6, 40_000
+    rows = k + 1
+    tgt1 = (1.5 * rng.normal(size=(1, rows, V))).astype(np.float32)
+    drf1 = (tgt1 + 1.0 * rng.normal(size=(1, rows, V))).astype(np.float32)[:, :k]
+    tgt, drf = np.repeat(tgt1, B, axis=0), np.repeat(drf1, B, axis=0)
+    t_row = np.array([0.4, 2.5, 1.0], np.float32)
+    temps = np.repeat(t_row[None, :], B, axis=0)
+    out = oracle.verify(tgt, drf, np.arange(B, dtype=np.uint64) + 3, T=1.0, temps=temps)
+    m = [match_closed_form(softmax(tgt1[0, j], float(t_row[j])), softmax(drf1[0, j], float(t_row[j]))) for j in range(k)]
+    m_swapped = [match_closed_form(softmax(tgt1[0, j], float(t_row[1 - j])), softmax(drf1[0, j], float(t_row[1 - j]))) for j in range(k)]
+    hit = out["draft_tok"] == out["target_tok"][:, :k]
+    for j in range(k):
+        sd = math.sqrt(m[j] * (1 - m[j]) / B)
+        assert abs(hit[:, j].mean() - m[j]) < 4.5 * sd, (j, hit[:, j].mean(), m[j])
+        assert abs(hit[:, j].mean() - m_swapped[j]) > 8 * sd   # the pin can tell the rows apart
