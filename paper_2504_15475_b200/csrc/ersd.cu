@@ -161,7 +161,9 @@ static size_t workspace_bytes(int64_t B, int64_t rows) {
   return (size_t)B * (size_t)rows * sizeof(Slot);
 }
 
-static int get_workspace(const ersd_opts& o, size_t need, void** ws) {
+// The private workspace of a device is zeroed on the stream of the call that (re)allocates it, so
+// that the zeroing is ordered before that call's kernel whatever kind of stream it is.
+static int get_workspace(const ersd_opts& o, size_t need, void** ws, cudaStream_t stream) {
   if (o.workspace) {
     if (o.workspace_bytes < need) return ERSD_EWORKSPACE;
     if (((uintptr_t)o.workspace & 15) != 0) return ERSD_EALIGN;
@@ -187,7 +189,7 @@ static int get_workspace(const ersd_opts& o, size_t need, void** ws) {
       w.ptr = nullptr;
       return cuda_fail(e);
     }
-    e = cudaMemset(w.ptr, 0, grow);
+    e = cudaMemsetAsync(w.ptr, 0, grow, stream);
     if (e != cudaSuccess) return cuda_fail(e);
     w.bytes = grow;
   }
@@ -216,10 +218,28 @@ static bool rows_aligned(const void* base, int64_t ld, int dt) {
 
 constexpr int kMinChunkTiles = 8;  // smallest chunk of a row that the default split makes
 
+// Multiprocessors of the current device (asked once per device; 148 on a B200).
+static int sm_count() {
+  static std::mutex m;
+  static int count[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  std::lock_guard<std::mutex> lock(m);
+  if (!count[dev]) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) {
+      (void)cudaGetLastError();
+      n = 148;
+    }
+    count[dev] = n;
+  }
+  return count[dev];
+}
+
 // Block size of a call: opts->block_threads if given, else 128-thread blocks when there are enough
 // rows to give every one of their (twice as many) resident-block slots a chunk, 256 otherwise.
 static int choose_threads(const ersd_opts& o, int64_t units, int* threads) {
-  if (o.block_threads == 0) *threads = units >= 148 * b128::kMinBlocks ? 128 : 256;
+  if (o.block_threads == 0) *threads = units >= (int64_t)sm_count() * b128::kMinBlocks ? 128 : 256;
   else if (o.block_threads == 128 || o.block_threads == 256) *threads = (int)o.block_threads;
   else return ERSD_EINVAL;
   return ERSD_OK;
@@ -240,7 +260,7 @@ static int choose_split(const ersd_opts& o, int64_t units, int V, int cmax, int 
     S = (int)o.split_v;
     if (S > ntiles) S = ntiles;
   } else {
-    const int64_t slots = 148 * (threads == 128 ? b128::kMinBlocks : b256::kMinBlocks);
+    const int64_t slots = (int64_t)sm_count() * (threads == 128 ? b128::kMinBlocks : b256::kMinBlocks);
     S = (int)((slots + units - 1) / units);
     if (S < 2 && (int64_t)ntiles * tile >= 4 * kMinChunkTiles * b256::kTile) S = 2;
     const int by_v = ntiles / kMinChunkTiles;
@@ -333,7 +353,7 @@ static int prefer_shared_memory() {
 // block's decided indices (measured: a star of 8 at B=1 48 -> 42 us, the 17-node tree 35 -> 33 us;
 // at 544 rows the pooling costs 0.7 % instead).
 static int launch(const Params& p, const TreeDesc& tree, int dt, bool many, cudaStream_t st) {
-  many = many && (int64_t)p.B * p.rows <= 2 * 148;
+  many = many && (int64_t)p.B * p.rows <= 2 * sm_count();
   // grid (sequence, row in launch order, chunk): blocks are dispatched x fastest, z slowest, which
   // is the chunk-major order the kernel counts on, and the kernel needs no division to decode
   if (p.rows > 65535 || p.S > 65535) return ERSD_EUNSUPPORTED;
@@ -461,7 +481,7 @@ static int cluster_size(const ersd_opts& o, const Params& p, int dt, int* out) {
   int CL = 1;
   while (CL < lim && CL * b256::kClusterGroups < ntiles) CL *= 2;
   const int64_t units = (int64_t)p.B * p.rows;
-  if (units * CL > 2 * 148 && CL > 1 && (CL / 2) * 2 * b256::kClusterGroups >= ntiles &&
+  if (units * CL > 2 * sm_count() && CL > 1 && (CL / 2) * 2 * b256::kClusterGroups >= ntiles &&
       (ntiles + CL / 2 - 1) / (CL / 2) <= max_tiles)
     CL /= 2;
   *out = CL;
@@ -537,7 +557,8 @@ static void fill_common(Params& p, const ersd_opts& o, const uint64_t* seeds, in
 static int verify_impl(const void* target, const void* draft, int dt, const TreeDesc& tree, int D,
                        int cmax, bool chain, const uint64_t* seeds, int B, int rows, int draft_rows,
                        int V, float T, int32_t* out_tokens, int32_t* out_accept_len,
-                       const ersd_opts* opts, void* stream, const int32_t* given_tok = nullptr) {
+                       const ersd_opts* opts, void* stream, const int32_t* given_tok = nullptr,
+                       bool check_only = false) {
   const ersd_opts o = read_opts(opts);
   Params p;
   memset(&p, 0, sizeof p);
@@ -566,8 +587,14 @@ static int verify_impl(const void* target, const void* draft, int dt, const Tree
   if (o.kernel_path > 2) return ERSD_EINVAL;
   const bool cluster_ok = cmax <= 1 && cluster_applies(p, dt);  // (a tree without branching is the chain 0 -> 1 -> ...)
   if (o.kernel_path == 2 && !cluster_ok) return ERSD_EUNSUPPORTED;
+  if (o.block_threads != 0 && o.block_threads != 128 && o.block_threads != 256) return ERSD_EINVAL;
+  if (o.workspace) {
+    if (o.workspace_bytes < workspace_bytes(B, rows)) return ERSD_EWORKSPACE;
+    if (((uintptr_t)o.workspace & 15) != 0) return ERSD_EALIGN;
+  }
+  if (check_only) return ERSD_OK;  // every host-side check has passed; nothing was enqueued
   void* ws = nullptr;
-  const int st = get_workspace(o, workspace_bytes(B, rows), &ws);
+  const int st = get_workspace(o, workspace_bytes(B, rows), &ws, (cudaStream_t)stream);
   if (st != ERSD_OK) return st;
   p.slots = (Slot*)ws;
   if (cluster_ok && (o.kernel_path == 2 || cluster_by_default(o, p, dt)))
@@ -641,7 +668,7 @@ int ersd_race_sample(const void* logits, ersd_dtype dt, const uint64_t* seeds, i
   set_chunks(p, choose_split(o, (int64_t)B * R, V, c, p.threads));
   if (p.S > 1) {
     void* ws = nullptr;
-    st = get_workspace(o, workspace_bytes(B, R), &ws);
+    st = get_workspace(o, workspace_bytes(B, R), &ws, (cudaStream_t)cuda_stream);
     if (st != ERSD_OK) return st;
     p.slots = (Slot*)ws;
   }
@@ -650,9 +677,10 @@ int ersd_race_sample(const void* logits, ersd_dtype dt, const uint64_t* seeds, i
   return launch(p, tree, dt, c > 1, (cudaStream_t)cuda_stream);
 }
 
-int ersd_verify(const void* target_logits, const void* draft_logits, ersd_dtype dt,
-                const uint64_t* seeds, int B, int k, int V, float T, int32_t* out_tokens,
-                int32_t* out_accept_len, const ersd_opts* opts, void* cuda_stream) {
+static int verify_sequence(const void* target_logits, const void* draft_logits, int dt,
+                           const uint64_t* seeds, int B, int k, int V, float T, int32_t* out_tokens,
+                           int32_t* out_accept_len, const ersd_opts* opts, void* cuda_stream,
+                           bool check_only) {
   if (k < 0) return ERSD_EINVAL;
   if (k + 1 > ERSD_MAX_ROWS) return ERSD_EUNSUPPORTED;
   int st = check_common(target_logits, dt, seeds, B, k + 1, V, T);
@@ -669,7 +697,14 @@ int ersd_verify(const void* target_logits, const void* draft_logits, ersd_dtype 
   st = build_tree(parent, k, &tree, &D, &cmax);
   if (st != ERSD_OK) return st;
   return verify_impl(target_logits, draft_logits, dt, tree, D, cmax, true, seeds, B, k + 1, k, V, T,
-                     out_tokens, out_accept_len, opts, cuda_stream);
+                     out_tokens, out_accept_len, opts, cuda_stream, nullptr, check_only);
+}
+
+int ersd_verify(const void* target_logits, const void* draft_logits, ersd_dtype dt,
+                const uint64_t* seeds, int B, int k, int V, float T, int32_t* out_tokens,
+                int32_t* out_accept_len, const ersd_opts* opts, void* cuda_stream) {
+  return verify_sequence(target_logits, draft_logits, dt, seeds, B, k, V, T, out_tokens, out_accept_len,
+                         opts, cuda_stream, false);
 }
 
 int ersd_verify_tokens(const void* target_logits, const int32_t* draft_tokens, ersd_dtype dt,
@@ -728,18 +763,22 @@ int ersd_verify_noalloc(const void* target_logits, const void* draft_logits, ers
   ersd_opts o = read_opts(opts);
   if (o.workspace) return ERSD_EINVAL;  // this entry point brings its own scratch
   void* scratch = nullptr;
-  const int st = noalloc_scratch(&scratch);
+  int st = noalloc_scratch(&scratch);
+  if (st != ERSD_OK) return st;
+  o.struct_size = sizeof o;
+  o.workspace = scratch;
+  o.workspace_bytes = kNoallocBytes;
+  // every host-side argument check of ersd_verify first: a refused call puts nothing on the stream
+  st = verify_sequence(target_logits, draft_logits, dt, seeds, B, k, V, T, out_tokens, out_accept_len, &o,
+                       cuda_stream, true);
   if (st != ERSD_OK) return st;
   // The array keeps whatever the previous call left; the arrival counters (the first 16 bytes
   // of every slot this call uses) must start at zero.
   const cudaError_t e = cudaMemset2DAsync(scratch, sizeof(Slot), 0, 16, (size_t)B * ((size_t)k + 1),
                                           (cudaStream_t)cuda_stream);
   if (e != cudaSuccess) return cuda_fail(e);
-  o.struct_size = sizeof o;
-  o.workspace = scratch;
-  o.workspace_bytes = kNoallocBytes;
-  return ersd_verify(target_logits, draft_logits, dt, seeds, B, k, V, T, out_tokens, out_accept_len,
-                     &o, cuda_stream);
+  return verify_sequence(target_logits, draft_logits, dt, seeds, B, k, V, T, out_tokens, out_accept_len, &o,
+                         cuda_stream, false);
 }
 
 int ersd_tree_depth(const int32_t* parent, int N) {

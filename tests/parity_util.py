@@ -87,6 +87,20 @@ def check_verify(inp, out, seq_ids=None, pos_offsets=None):
     flips = int(d1.sum() + d2.sum())
     for b in range(B):
         if d1[b].any() or d2[b].any():
+            # near-tie in this sequence: the walk must be right for the winners the GPU chose
+            tt, dt = g["target_tok"][b], g["draft_tok"][b]
+            cur, toks, path = 0, [], []
+            while True:
+                toks.append(int(tt[cur]))
+                path.append(cur)
+                nxt = [m for m in range(1, nodes) if parent[m] == cur and tt[cur] >= 0 and dt[m] == tt[cur]]
+                if not nxt:
+                    break
+                cur = nxt[0]
+            L = len(toks) - 1
+            assert g["accept_len"][b] == L
+            assert list(g["tokens"][b, :L + 1]) == toks and (g["tokens"][b, L + 1:] == -1).all()
+            assert list(g["path"][b, :L + 1]) == path and (g["path"][b, L + 1:] == -1).all()
             continue
         assert g["accept_len"][b] == ref["accept_len"][b]
         assert (g["tokens"][b] == ref["tokens"][b]).all(), (b, g["tokens"][b], ref["tokens"][b])

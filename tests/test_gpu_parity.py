@@ -595,20 +595,27 @@ def test_workspace_reused_by_calls_of_different_sizes(ersd):
             w = wl.Workload("ws", B=B, k=k, V=V, dtype="bf16", sigma=0.8, T=1.0, config_id=48)
             inp = wl.make_inputs(w, call=n)
             d = to_dev(inp)
-            tok = torch.empty(B, k + 1, dtype=torch.int32, device="cuda")
-            acc = torch.empty(B, dtype=torch.int32, device="cuda")
-            ersd.ersd_verify(d["target"], d["draft"] if k else None, d["seeds"], 1.0, tok, acc,
-                             ersd.make_opts(workspace=ws, split_v=(0, 2)[rnd]))
+            out = dict(tokens=torch.empty(B, k + 1, dtype=torch.int32, device="cuda"),
+                       accept_len=torch.empty(B, dtype=torch.int32, device="cuda"),
+                       draft_tok=torch.empty(B, k, dtype=torch.int32, device="cuda"),
+                       draft_key=torch.empty(B, k, dtype=torch.float32, device="cuda"),
+                       target_tok=torch.empty(B, k + 1, dtype=torch.int32, device="cuda"),
+                       target_key=torch.empty(B, k + 1, dtype=torch.float32, device="cuda"))
+            ersd.ersd_verify(d["target"], d["draft"] if k else None, d["seeds"], 1.0, out["tokens"],
+                             out["accept_len"],
+                             ersd.make_opts(workspace=ws, split_v=(0, 2)[rnd], out_draft_tok=out["draft_tok"],
+                                            out_draft_key=out["draft_key"], out_target_tok=out["target_tok"],
+                                            out_target_key=out["target_key"]))
             torch.cuda.synchronize()
-            import oracle
             if k:
-                ref = oracle.verify(wl.as_numpy_logits(inp["target"]), wl.as_numpy_logits(inp["draft"]),
-                                    wl.seeds_as_u64(inp["seeds"]), T=1.0)
-                if min((ref["target_key"][..., 1] - ref["target_key"][..., 0]).min(),
-                       (ref["draft_key"][..., 1] - ref["draft_key"][..., 0]).min()) < 1e-5:
-                    continue
-                assert (tok.cpu().numpy() == ref["tokens"]).all(), (rnd, n)
-                assert (acc.cpu().numpy() == ref["accept_len"]).all(), (rnd, n)
+                check_verify(inp, out)     # near-tie rows may take either winner; nothing is skipped
+            else:
+                ref_tok, ref_key = __import__("oracle").race_sample(
+                    wl.as_numpy_logits(inp["target"]), wl.seeds_as_u64(inp["seeds"]), T=1.0)
+                got = out["target_tok"].cpu().numpy()
+                near = (ref_key[..., 1] - ref_key[..., 0]) < 1e-5
+                assert ((got == ref_tok[..., 0]) | near).all(), (rnd, n)
+                assert (out["accept_len"].cpu().numpy() == 0).all()
 
 
 def test_host_buffer_entry(ersd):
