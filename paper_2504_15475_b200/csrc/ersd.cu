@@ -96,7 +96,7 @@ constexpr bool kMany = false;
 #include "ersd_kernel.inc"
 }  // namespace b256
 namespace b128 {
-constexpr int kThreads = 128, kMinBlocks = 8;
+constexpr int kThreads = 128, kMinBlocks = 7;
 constexpr bool kMany = false;
 #include "ersd_kernel.inc"
 }  // namespace b128
@@ -107,7 +107,7 @@ constexpr bool kMany = true;
 #include "ersd_kernel.inc"
 }  // namespace b256m
 namespace b128m {
-constexpr int kThreads = 128, kMinBlocks = 8;
+constexpr int kThreads = 128, kMinBlocks = 7;
 constexpr bool kMany = true;
 #include "ersd_kernel.inc"
 }  // namespace b128m
@@ -832,6 +832,6 @@ const char* ersd_status_string(int status) {
 
 int ersd_last_cuda_error(void) { return g_last_cuda_error; }
 
-int ersd_version(void) { return 108; }
+int ersd_version(void) { return 109; }
 
 }  // extern "C"
