@@ -43,10 +43,17 @@
  *     every verify call, exchange partial results through a workspace.  Give
  *     one in opts->workspace (size from ersd_workspace_bytes, zeroed once
  *     with ersd_workspace_init; every call leaves it ready for the next
- *     call, of any size that fits) or pass none
- *     and the library keeps a private one per device, (re)allocated with
- *     cudaMalloc when a call needs more than it holds.  Two calls that may
- *     overlap on the GPU must not share a workspace.
+ *     call, of any size that fits): then the call allocates nothing and only
+ *     enqueues work on `cuda_stream`.  Or pass none and the library keeps ONE
+ *     private workspace per device.  Two things follow from that.  (1) A call
+ *     that needs more than the private workspace holds makes it grow with
+ *     cudaFree and cudaMalloc, which synchronise the whole device, and zeroes
+ *     it on `cuda_stream`; such a call is not asynchronous and cannot be part
+ *     of a stream capture.  (2) Every call on the device that passes no
+ *     workspace uses that same memory, whatever its stream: such calls must
+ *     not overlap on the GPU.  Calls that may overlap (different streams,
+ *     host threads without ordering between them) each need a workspace of
+ *     their own in opts->workspace; sharing one gives wrong results.
  *   - Randomness contract: a (seed, sequence id, position) triple must not be
  *     reused for two EMITTED tokens.  Reusing the positions of a rejected
  *     speculation in the next round is fine: what is emitted depends only on
@@ -112,6 +119,14 @@ typedef struct ersd_opts {
                               blocks to stage in shared memory: beyond about 320 k entries in bf16,
                               160 k in fp32, halved when draft rows are raced along) */
   uint32_t reserved1;
+  uint32_t* near_tie_count; /* device, nullable: a counter the call ADDS to (the caller zeroes it): the number
+                              of races in which two consecutive arrivals among the first c + 1 (c = arrivals
+                              wanted: 1 for a winner, a node's child count for its draft row, top_c) have race
+                              keys closer than 1e-5 -- the benchmark spec's near-tie window, inside which a reference
+                              in other arithmetic may order the two the other way.  To see the runner-up every
+                              race is run for one more arrival (c + 1 <= ERSD_MAX_TOP_C, else
+                              ERSD_EUNSUPPORTED), which costs time, and the call takes the streaming kernel
+                              (kernel_path 2 is refused).  Leave NULL in production. */
 } ersd_opts;
 
 /*
@@ -125,8 +140,11 @@ typedef struct ersd_opts {
  *   logits  device [B, R, V] of dtype dt       seeds   device [B] uint64
  *   out_tok device [B, R, c] int32
  * Errors: ERSD_EINVAL for null pointers, B, R, V < 1 or B * R beyond 2^31 - 1,
- * T < 0 or not finite; ERSD_EUNSUPPORTED for c > ERSD_MAX_TOP_C or
- * V > 0x7FFF0000; ERSD_EALIGN.
+ * T < 0 or not finite; ERSD_EUNSUPPORTED for c > ERSD_MAX_TOP_C,
+ * V > 0x7FFF0000, or more than 65535 rows per sequence or thread blocks per
+ * row (the launch grid is (B, rows, blocks per row); fold rows into B -- with
+ * opts->seq_ids and opts->pos_offsets naming each row's race -- to sample more
+ * rows of one sequence in a call); ERSD_EALIGN.
  */
 int ersd_race_sample(const void* logits, ersd_dtype dt, const uint64_t* seeds, int B, int R, int V,
                      float T, int32_t* out_tok, const ersd_opts* opts, void* cuda_stream);

@@ -45,6 +45,8 @@ def lib():
         _lib.ersd_oracle_token_word.restype = C.c_uint32
         _lib.ersd_oracle_token_word.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32]
         _lib.ersd_oracle_max_threads.restype = C.c_int
+        _lib.ersd_oracle_gsd_uniform.restype = C.c_double
+        _lib.ersd_oracle_gsd_uniform.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32]
     return _lib
 
 
@@ -260,4 +262,64 @@ def verify_tree(target: np.ndarray, draft: np.ndarray, parent, seeds, T: float =
         C.c_int(V), C.c_float(float(T)), _p(temps), C.c_int64(nodes), C.c_int64(1), C.c_int(D),
         C.c_int(max_c), _p(out["tokens"]), _p(out["accept_len"]), _p(out["path"]),
         _p(out["arrivals"]), _p(out["target_tok"]), _p(out["arrival_key"]), _p(out["target_key"]))
+    return out
+
+
+def gsd_uniform(seed: int, seq_id: int, node: int, rank: int = 0) -> float:
+    """The uniform of the ratio test of child `rank` of node (or position) `node`."""
+    return float(lib().ersd_oracle_gsd_uniform(C.c_uint64(int(seed)), C.c_uint32(int(seq_id)),
+                                               C.c_uint32(int(node)), C.c_uint32(int(rank))))
+
+
+def gsd_verify(target: np.ndarray, draft: np.ndarray, draft_tokens, seeds, T: float = 1.0, temps=None,
+               seq_ids=None, pos_offsets=None):
+    """Sequence GSD (Algorithm 1 position by position).  target [B, k+1, V], draft [B, k, V],
+    draft_tokens [B, k] -> dict(tokens [B, k+1] (-1 padded), accept_len [B], ratio, unif [B, k],
+    last_times [B, 2])."""
+    target = np.ascontiguousarray(target)
+    draft = np.ascontiguousarray(draft)
+    B, rows, V = target.shape
+    k = rows - 1
+    assert draft.shape == (B, k, V) and draft.dtype == target.dtype
+    tok = np.ascontiguousarray(draft_tokens, dtype=np.int32)
+    assert tok.shape == (B, k)
+    seeds = np.ascontiguousarray(seeds, dtype=np.uint64)
+    temps = _opt(temps, np.float32)
+    if temps is not None:
+        assert temps.shape == (B, rows)
+    seq_ids = _opt(seq_ids, np.uint32)
+    pos_offsets = _opt(pos_offsets, np.uint32)
+    out = dict(tokens=np.empty((B, rows), np.int32), accept_len=np.empty(B, np.int32),
+               ratio=np.empty((B, k), np.float64), unif=np.empty((B, k), np.float64),
+               last_times=np.full((B, 2), np.inf))
+    lib().ersd_oracle_gsd_verify(
+        _p(target), _p(draft), _p(tok), C.c_int(_dtype_of(target)), _p(seeds), _p(seq_ids), _p(pos_offsets),
+        C.c_int(B), C.c_int(k), C.c_int(V), C.c_float(float(T)), _p(temps), C.c_int64(rows), C.c_int64(1),
+        _p(out["tokens"]), _p(out["accept_len"]), _p(out["ratio"]), _p(out["unif"]), _p(out["last_times"]))
+    return out
+
+
+def gsd_verify_tree(target: np.ndarray, draft: np.ndarray, draft_tokens, parent, seeds, T: float = 1.0,
+                    temps=None, seq_ids=None, pos_offsets=None):
+    """Tree GSD (Algorithm 4).  target, draft [B, N+1, V]; draft_tokens [B, N+1] (entry 0 unused);
+    parent [N+1] -> dict(tokens [B, D+1], accept_len [B], path [B, D+1], last_times [B, 2])."""
+    target = np.ascontiguousarray(target)
+    draft = np.ascontiguousarray(draft)
+    B, nodes, V = target.shape
+    assert draft.shape == target.shape and draft.dtype == target.dtype
+    parent = np.ascontiguousarray(parent, dtype=np.int32)
+    D, _, _, _ = tree_shape(parent)
+    tok = np.ascontiguousarray(draft_tokens, dtype=np.int32)
+    assert tok.shape == (B, nodes)
+    seeds = np.ascontiguousarray(seeds, dtype=np.uint64)
+    temps = _opt(temps, np.float32)
+    seq_ids = _opt(seq_ids, np.uint32)
+    pos_offsets = _opt(pos_offsets, np.uint32)
+    out = dict(tokens=np.empty((B, D + 1), np.int32), accept_len=np.empty(B, np.int32),
+               path=np.empty((B, D + 1), np.int32), last_times=np.full((B, 2), np.inf), depth=D)
+    lib().ersd_oracle_gsd_verify_tree(
+        _p(target), _p(draft), _p(tok), C.c_int(_dtype_of(target)), _p(parent), _p(seeds), _p(seq_ids),
+        _p(pos_offsets), C.c_int(B), C.c_int(nodes - 1), C.c_int(V), C.c_float(float(T)), _p(temps),
+        C.c_int64(nodes), C.c_int64(1), C.c_int(D), _p(out["tokens"]), _p(out["accept_len"]), _p(out["path"]),
+        _p(out["last_times"]))
     return out

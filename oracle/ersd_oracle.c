@@ -371,3 +371,219 @@ int ersd_oracle_max_threads(void) {
   return 1;
 #endif
 }
+
+/* ================================================================== */
+/* Greedy speculative decoding (GSD): Algorithm 1 (Section 2) and its  */
+/* tree form, Algorithm 4 (Appendix A).  The comparison verifier of    */
+/* the paper: a ratio test per drafted token and, on rejection, a      */
+/* sample of the residual law max(P - Q, 0) / sum.                      */
+/*                                                                      */
+/* What the paper leaves open and this build fixes: the uniform of a    */
+/* ratio test is word 0 of Philox4x32-10 with counter (child rank,      */
+/* node or position, sequence id, 1), u = (x + 1/2) 2^-32; the token    */
+/* that ends the call (residual sample, or the sample of the last       */
+/* target row when everything was accepted) is the winner of an         */
+/* exponential race (exact by Section 3) whose variables come from      */
+/* counter (i >> 2, node or position, sequence id, 2) -- streams        */
+/* separate from the one that drafting uses (last counter word 0), as   */
+/* Algorithm 1 needs the residual sample independent of the draft.      */
+/* Algorithm 4 is garbled in two places (the tested token is typeset    */
+/* without its child index, and an empty loop follows the inner while): */
+/* the reading taken is the one of Section 2's text -- at each vertex    */
+/* the children are tried in order, each rejection replaces the target  */
+/* law by its normalised residual against the current draft law and     */
+/* removes the rejected token from the draft law (sampling without      */
+/* replacement), an acceptance moves to that child.                     */
+/* ================================================================== */
+
+static double gsd_uniform(uint64_t seed, uint32_t seq_id, uint32_t node, uint32_t rank) {
+  uint32_t ctr[4] = {rank, node, seq_id, 1u};
+  uint32_t key[2] = {(uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32)};
+  uint32_t out[4];
+  ersd_oracle_philox4x32_10(ctr, key, out);
+  return ((double)out[0] + 0.5) * (1.0 / 4294967296.0);
+}
+
+double ersd_oracle_gsd_uniform(uint64_t seed, uint32_t seq_id, uint32_t node, uint32_t rank) {
+  return gsd_uniform(seed, seq_id, node, rank);
+}
+
+static double gsd_race_variate(uint64_t seed, uint32_t seq_id, uint32_t node, uint32_t i) {
+  uint32_t ctr[4] = {i >> 2, node, seq_id, 2u};
+  uint32_t key[2] = {(uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32)};
+  uint32_t out[4];
+  ersd_oracle_philox4x32_10(ctr, key, out);
+  return ersd_oracle_exp_variate(out[i & 3u]);
+}
+
+/* p = softmax(z / T) in double precision, maximum subtracted. */
+static void softmax_row(const void* row, int dtype, int V, double T, double* p) {
+  double zmax = -INFINITY, Z = 0.0;
+  for (int i = 0; i < V; ++i) {
+    double s = logit_at(row, dtype, i) / T;
+    if (s > zmax) zmax = s;
+  }
+  for (int i = 0; i < V; ++i) {
+    p[i] = exp(logit_at(row, dtype, i) / T - zmax);
+    Z += p[i];
+  }
+  for (int i = 0; i < V; ++i) p[i] /= Z;
+}
+
+/* Winner of the exponential race over non-negative weights w (argmin e_i / w_i over w_i > 0,
+ * ties to the lowest id), with the GSD race stream of `node`; -1 if no weight is positive.
+ * times[0], times[1] receive the winner's and the runner-up's arrival time. */
+static int32_t gsd_race(const double* w, int V, uint64_t seed, uint32_t seq_id, uint32_t node,
+                        double* times) {
+  double best = INFINITY, second = INFINITY;
+  int32_t arg = -1;
+  for (int i = 0; i < V; ++i) {
+    if (!(w[i] > 0.0)) continue;
+    double t = gsd_race_variate(seed, seq_id, node, (uint32_t)i) / w[i];
+    if (t < best) {
+      second = best;
+      best = t;
+      arg = i;
+    } else if (t < second) {
+      second = t;
+    }
+  }
+  if (times) {
+    times[0] = best;
+    times[1] = second;
+  }
+  return arg;
+}
+
+/* Sequence GSD (Algorithm 1, applied position by position as Section 2 describes: drafted
+ * tokens are verified in order until the first rejection).
+ *   draft_tok[b, j]   the token drafted at position j (a sample of draft row j, made earlier)
+ *   accept position j iff P_j(x) / Q_j(x) > u_j; at the first rejection emit a sample of
+ *   max(P_j - Q_j, 0) / sum and stop; after k acceptances emit a sample of target row k.
+ *   out_tokens [B, k+1] (-1 padded), out_accept_len [B];
+ *   ratio, unif [B, k]: the tested ratio and uniform of every position that was tested (NaN
+ *   elsewhere); last_times [B, 2]: arrival times of the final race's winner and runner-up. */
+void ersd_oracle_gsd_verify(const void* target, const void* draft, const int32_t* draft_tok,
+                            int dtype, const uint64_t* seeds, const uint32_t* seq_ids,
+                            const uint32_t* pos_offsets, int B, int k, int V, float T,
+                            const float* temps, int64_t temp_sb, int64_t temp_sr,
+                            int32_t* out_tokens, int32_t* out_accept_len, double* ratio,
+                            double* unif, double* last_times) {
+  int rows = k + 1;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int b = 0; b < B; ++b) {
+    double* p = (double*)malloc(sizeof(double) * (size_t)V);
+    double* q = (double*)malloc(sizeof(double) * (size_t)V);
+    uint32_t seq = seq_ids ? seq_ids[b] : (uint32_t)b;
+    uint32_t pos0 = pos_offsets ? pos_offsets[b] : 0u;
+    int32_t* y = out_tokens + (int64_t)b * rows;
+    for (int j = 0; j < rows; ++j) y[j] = -1;
+    for (int j = 0; j < k; ++j) {
+      ratio[(int64_t)b * k + j] = NAN;
+      unif[(int64_t)b * k + j] = NAN;
+    }
+    int L = 0, done = 0;
+    for (int j = 0; j < k && !done; ++j) {
+      double Tj = temp_of(T, temps, temp_sb, temp_sr, b, j);
+      softmax_row(row_ptr(target, dtype, ((int64_t)b * rows + j) * V), dtype, V, Tj, p);
+      softmax_row(row_ptr(draft, dtype, ((int64_t)b * k + j) * V), dtype, V, Tj, q);
+      int32_t x = draft_tok[(int64_t)b * k + j];
+      double u = gsd_uniform(seeds[b], seq, pos0 + (uint32_t)j, 0u);
+      double r = (x >= 0 && x < V) ? p[x] / q[x] : 0.0; /* 0/0: a token neither law can emit is rejected */
+      if (!(r == r)) r = 0.0;
+      ratio[(int64_t)b * k + j] = r;
+      unif[(int64_t)b * k + j] = u;
+      if (r > u) {
+        y[j] = x;
+        ++L;
+      } else {
+        for (int i = 0; i < V; ++i) p[i] = (p[i] > q[i]) ? p[i] - q[i] : 0.0; /* residual, unnormalised: the race is scale free */
+        y[j] = gsd_race(p, V, seeds[b], seq, pos0 + (uint32_t)j, last_times + 2 * (int64_t)b);
+        done = 1;
+      }
+    }
+    if (!done) {
+      double Tk = temp_of(T, temps, temp_sb, temp_sr, b, k);
+      softmax_row(row_ptr(target, dtype, ((int64_t)b * rows + k) * V), dtype, V, Tk, p);
+      y[k] = gsd_race(p, V, seeds[b], seq, pos0 + (uint32_t)k, last_times + 2 * (int64_t)b);
+    }
+    out_accept_len[b] = L;
+    free(p);
+    free(q);
+  }
+}
+
+/* Tree GSD (Algorithm 4).  Nodes 0..N, node 0 the root, parent[n] < n, siblings ordered by node
+ * id; draft_tok[b, n] is the token drafted at node n (node 0: unused), siblings drafted without
+ * replacement from their parent's draft row.  Walk from the root: try the current node's
+ * children in order -- child of rank i is accepted iff P_t(x) / Q_d(x) > u(node, i), where after
+ * every rejection P_t <- max(P_t - Q_d, 0) / sum and Q_d <- Q_d with the rejected token removed,
+ * renormalised -- move to an accepted child; when no child is accepted (or there is none) emit
+ * a sample of the current P_t and stop.
+ *   out_tokens [B, D+1] (-1 padded), out_accept_len [B], out_path [B, D+1] (node ids). */
+void ersd_oracle_gsd_verify_tree(const void* target, const void* draft, const int32_t* draft_tok,
+                                 int dtype, const int32_t* parent, const uint64_t* seeds,
+                                 const uint32_t* seq_ids, const uint32_t* pos_offsets, int B, int N,
+                                 int V, float T, const float* temps, int64_t temp_sb,
+                                 int64_t temp_sr, int D, int32_t* out_tokens,
+                                 int32_t* out_accept_len, int32_t* out_path, double* last_times) {
+  int nodes = N + 1;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int b = 0; b < B; ++b) {
+    double* p = (double*)malloc(sizeof(double) * (size_t)V);
+    double* q = (double*)malloc(sizeof(double) * (size_t)V);
+    uint32_t seq = seq_ids ? seq_ids[b] : (uint32_t)b;
+    uint32_t pos0 = pos_offsets ? pos_offsets[b] : 0u;
+    int32_t* y = out_tokens + (int64_t)b * (D + 1);
+    int32_t* path = out_path + (int64_t)b * (D + 1);
+    for (int d = 0; d <= D; ++d) {
+      y[d] = -1;
+      path[d] = -1;
+    }
+    int cur = 0, depth = 0;
+    for (;;) {
+      double Tn = temp_of(T, temps, temp_sb, temp_sr, b, cur);
+      softmax_row(row_ptr(target, dtype, ((int64_t)b * nodes + cur) * V), dtype, V, Tn, p);
+      int have_q = 0, next = -1;
+      uint32_t rank = 0;
+      for (int m = cur + 1; m < nodes && next < 0; ++m) {
+        if (parent[m] != cur) continue;
+        if (!have_q) {
+          softmax_row(row_ptr(draft, dtype, ((int64_t)b * nodes + cur) * V), dtype, V, Tn, q);
+          have_q = 1;
+        }
+        int32_t x = draft_tok[(int64_t)b * nodes + m];
+        double u = gsd_uniform(seeds[b], seq, pos0 + (uint32_t)cur, rank);
+        double r = (x >= 0 && x < V) ? p[x] / q[x] : 0.0;
+        if (!(r == r)) r = 0.0;
+        if (r > u) {
+          next = m;
+          y[depth] = x;
+        } else {
+          double sp = 0.0, sq = 0.0;
+          for (int i = 0; i < V; ++i) {
+            p[i] = (p[i] > q[i]) ? p[i] - q[i] : 0.0;
+            sp += p[i];
+          }
+          if (sp > 0.0)
+            for (int i = 0; i < V; ++i) p[i] /= sp;
+          if (x >= 0 && x < V) q[x] = 0.0;
+          for (int i = 0; i < V; ++i) sq += q[i];
+          if (sq > 0.0)
+            for (int i = 0; i < V; ++i) q[i] /= sq;
+        }
+        ++rank;
+      }
+      path[depth] = cur;
+      if (next < 0) {
+        y[depth] = gsd_race(p, V, seeds[b], seq, pos0 + (uint32_t)cur, last_times + 2 * (int64_t)b);
+        break;
+      }
+      cur = next;
+      ++depth;
+    }
+    out_accept_len[b] = depth;
+    free(p);
+    free(q);
+  }
+}

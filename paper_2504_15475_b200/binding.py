@@ -39,6 +39,7 @@ class ErsdOpts(C.Structure):
         ("out_path", C.c_void_p), ("out_key", C.c_void_p),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
         ("kernel_path", C.c_uint32), ("reserved1", C.c_uint32),
+        ("near_tie_count", C.c_void_p),
     ]
 
 
@@ -132,7 +133,7 @@ def make_opts(*, top_c: int = 0, split_v: int = 0, block_threads: int = 0, ld_ta
               seq_ids: Optional[torch.Tensor] = None, pos_offsets: Optional[torch.Tensor] = None,
               out_draft_tok=None, out_draft_key=None, out_target_tok=None, out_target_key=None,
               out_path=None, out_key=None, workspace: Optional[torch.Tensor] = None,
-              kernel_path: int = 0) -> ErsdOpts:
+              kernel_path: int = 0, near_tie_count: Optional[torch.Tensor] = None) -> ErsdOpts:
     o = ErsdOpts()
     o.struct_size = C.sizeof(ErsdOpts)
     o.top_c, o.split_v, o.block_threads = top_c, split_v, block_threads
@@ -156,6 +157,8 @@ def make_opts(*, top_c: int = 0, split_v: int = 0, block_threads: int = 0, ld_ta
     if workspace is not None:
         o.workspace = workspace.data_ptr()
         o.workspace_bytes = workspace.numel() * workspace.element_size()
+    if near_tie_count is not None:  # int32 tensor of one element that the call adds to
+        o.near_tie_count = _dev(near_tie_count, torch.int32, "near_tie_count").data_ptr()
     return o
 
 

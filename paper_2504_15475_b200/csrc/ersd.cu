@@ -82,6 +82,8 @@ struct Params {
   int32_t* out_target_tok;
   float* out_target_key;
   float* out_key;        // sample mode
+  uint32_t* near_tie;    // count of races with two consecutive arrivals closer than 1e-5 (nullable)
+  int extra;             // 1 when near-ties are counted: every race is run for one more arrival
   Slot* slots;
 };
 
@@ -583,7 +585,13 @@ static int verify_impl(const void* target, const void* draft, int dt, const Tree
   p.out_draft_key = o.out_draft_key;
   p.out_target_tok = o.out_target_tok;
   p.out_target_key = o.out_target_key;
-  // sequences of few rows: one cluster per position (chains only: one arrival per race)
+  p.near_tie = o.near_tie_count;
+  p.extra = o.near_tie_count ? 1 : 0;
+  if (((uintptr_t)o.near_tie_count & 3) != 0) return ERSD_EALIGN;
+  if (cmax + p.extra > ERSD_MAX_TOP_C) return ERSD_EUNSUPPORTED;
+  cmax += p.extra;
+  // sequences of few rows: one cluster per position (chains only: one arrival per race; near-ties
+  // are counted by the streaming kernel only, the cluster kernel keeps no runner-up key)
   if (o.kernel_path > 2) return ERSD_EINVAL;
   const bool cluster_ok = cmax <= 1 && cluster_applies(p, dt);  // (a tree without branching is the chain 0 -> 1 -> ...)
   if (o.kernel_path == 2 && !cluster_ok) return ERSD_EUNSUPPORTED;
@@ -647,6 +655,9 @@ int ersd_race_sample(const void* logits, ersd_dtype dt, const uint64_t* seeds, i
   const ersd_opts o = read_opts(opts);
   const int c = o.top_c > 1 ? (int)o.top_c : 1;
   if (c > ERSD_MAX_TOP_C) return ERSD_EUNSUPPORTED;
+  const int extra = o.near_tie_count ? 1 : 0;
+  if (c + extra > ERSD_MAX_TOP_C) return ERSD_EUNSUPPORTED;
+  if (((uintptr_t)o.near_tie_count & 3) != 0) return ERSD_EALIGN;
   Params p;
   memset(&p, 0, sizeof p);
   fill_common(p, o, seeds, B, R, V, T);
@@ -660,12 +671,16 @@ int ersd_race_sample(const void* logits, ersd_dtype dt, const uint64_t* seeds, i
   p.aligned_d = 1;
   p.out_tokens = out_tok;
   p.out_key = o.out_key;
+  p.near_tie = o.near_tie_count;
+  p.extra = extra;
   if (o.kernel_path > 2) return ERSD_EINVAL;
-  if (o.kernel_path == 2 && !cluster_applies(p, dt)) return ERSD_EUNSUPPORTED;
-  if (o.kernel_path == 2 || cluster_by_default(o, p, dt)) return launch_cluster(o, p, dt, (cudaStream_t)cuda_stream);
+  // (near-ties are counted by the streaming kernel only: the cluster kernel keeps no runner-up key)
+  const bool cluster_ok = !extra && cluster_applies(p, dt);
+  if (o.kernel_path == 2 && !cluster_ok) return ERSD_EUNSUPPORTED;
+  if (cluster_ok && (o.kernel_path == 2 || cluster_by_default(o, p, dt))) return launch_cluster(o, p, dt, (cudaStream_t)cuda_stream);
   st = choose_threads(o, (int64_t)B * R, &p.threads);
   if (st != ERSD_OK) return st;
-  set_chunks(p, choose_split(o, (int64_t)B * R, V, c, p.threads));
+  set_chunks(p, choose_split(o, (int64_t)B * R, V, c + extra, p.threads));
   if (p.S > 1) {
     void* ws = nullptr;
     st = get_workspace(o, workspace_bytes(B, R), &ws, (cudaStream_t)cuda_stream);
@@ -674,7 +689,7 @@ int ersd_race_sample(const void* logits, ersd_dtype dt, const uint64_t* seeds, i
   }
   TreeDesc tree;
   memset(&tree, 0, sizeof tree);
-  return launch(p, tree, dt, c > 1, (cudaStream_t)cuda_stream);
+  return launch(p, tree, dt, c + extra > 1, (cudaStream_t)cuda_stream);
 }
 
 static int verify_sequence(const void* target_logits, const void* draft_logits, int dt,

@@ -51,15 +51,58 @@ def test_config2_calls(ersd, call):
     check_verify(inp, out)
 
 
-def test_config2_many_calls_count_near_ties(ersd):
-    """Sixty of config 2's seeded calls (2400 target and 1920 draft rows): winners equal the
-    oracle's everywhere but at oracle-flagged near-ties, which are counted (expected about
-    1e-5 per row, so usually none here)."""
-    flips = 0
-    for call in range(100, 160):
-        inp = wl.make_inputs(wl.CONFIGS["c2"], call=call)
-        flips += check_verify(inp, run_verify(ersd, inp))
-    assert flips <= 2
+def closed_form_match(p, q):
+    """sum_i 1 / sum_j max(p_j / p_i, q_j / q_i) for one row, in O(V log V) by sorting on p / q."""
+    r = p / q
+    o = np.argsort(r)
+    ps, qs = p[o], q[o]
+    tail_p = np.cumsum(ps[::-1])[::-1]                      # sum of p_j over r_j >= r_i
+    head_q = np.concatenate([[0.0], np.cumsum(qs)[:-1]])    # sum of q_j over r_j < r_i
+    return float((1.0 / (tail_p / ps + head_q / qs)).sum())
+
+
+def test_config2_all_thousand_calls(ersd):
+    """Config 2 as stated: 1000 seeded verify calls (B=8, k=4, V=32000; 40000 target and 32000
+    draft rows).  Every row's winners and keys and every accepted prefix equal the oracle's; the
+    only exception allowed is an oracle-flagged near-tie row, and those are counted (about 1e-5
+    per row expected, i.e. around one in the whole run).  The library's own near-tie counter must
+    see the same rows.  The accepted first positions stay within 4.5 sigma of the sum of the rows'
+    closed-form match probabilities (Section 3's coupling)."""
+    flips, counted, oracle_near = 0, 0, 0
+    exp_sum, var_sum, got = 0.0, 0.0, 0
+    near = torch.zeros(1, dtype=torch.int32, device="cuda")
+    w = wl.CONFIGS["c2"]
+    for call in range(1000):
+        inp = wl.make_inputs(w, call=call)
+        out = run_verify(ersd, inp)
+        flips += check_verify(inp, out)
+        if call % 10 == 0:   # every tenth call again with the near-tie counter on (a slower path)
+            d = to_dev(inp)
+            tok = torch.empty_like(out["tokens"])
+            acc = torch.empty_like(out["accept_len"])
+            ersd.ersd_verify(d["target"], d["draft"], d["seeds"], d["T"], tok, acc, ersd.make_opts(near_tie_count=near))
+            assert (tok == out["tokens"]).all() and (acc == out["accept_len"]).all()
+            import oracle
+            ref = oracle.verify(wl.as_numpy_logits(inp["target"]), wl.as_numpy_logits(inp["draft"]),
+                                wl.seeds_as_u64(inp["seeds"]), T=inp["T"])
+            for key in ("target_key", "draft_key"):
+                gap = ref[key][..., 1] - ref[key][..., 0]
+                oracle_near += int((gap < 1e-5).sum())
+                assert not ((gap > 0.99e-5) & (gap < 1.01e-5)).any()   # (no gap on the window's edge in these inputs)
+        if call % 25 == 0:   # the closed form on a sample of calls: 40 x 8 first positions
+            got += int((out["accept_len"] >= 1).sum().item())
+            p = torch.softmax(inp["target"][:, 0].double(), -1).numpy()
+            q = torch.softmax(inp["draft"][:, 0].double(), -1).numpy()
+            for b in range(w.B):
+                m = closed_form_match(p[b], q[b])
+                exp_sum += m
+                var_sum += m * (1 - m)
+    counted = int(near.item())
+    print("config 2, 1000 calls: near-tie rows taken the other way: %d; near-tie races counted by the "
+          "library on 100 calls: %d (oracle: %d)" % (flips, counted, oracle_near))
+    assert flips <= 3
+    assert counted == oracle_near
+    assert abs(got - exp_sum) < 4.5 * math.sqrt(var_sum), (got, exp_sum)
 
 
 @pytest.mark.parametrize("sigma,T", wl.C3_SWEEP)
@@ -88,8 +131,11 @@ def test_config5_reduced_batch_per_sequence_temperatures(ersd):
     check_verify(inp, out)
 
 
-# ------------------------------------------------------------------ full size, sampled sequences
-def _full_size_sampled(ersd, name, sample, **kw):
+# ------------------------------------------------------------------ full size, every sequence
+def _full_size(ersd, name, **kw):
+    """One call at the configuration's stated size, in the launch configuration the benchmark
+    times (library defaults), every sequence compared with the oracle.  Returns (inputs, outputs,
+    near-tie rows taken the other way)."""
     w = wl.CONFIGS[name]
     inp = wl.make_inputs(w, device="cuda", **kw)
     out = ersd.verify(inp["target"], inp["draft"], inp["seeds"], inp["T"], temps=inp.get("temps"),
@@ -98,67 +144,60 @@ def _full_size_sampled(ersd, name, sample, **kw):
     L = out["accept_len"].cpu().numpy()
     tok = out["tokens"].cpu().numpy()
     tt = out["target_tok"].cpu().numpy()
-    B = w.B
     # properties that hold at any size
     D = tok.shape[1] - 1
     assert ((0 <= L) & (L <= D)).all()
     assert (tt >= 0).all() and (tt < w.V).all()
-    for b in range(B):
+    for b in range(w.B):
         assert (tok[b, :L[b] + 1] >= 0).all() and (tok[b, L[b] + 1:] == -1).all()
     if not w.is_tree:
         dt = out["draft_tok"].cpu().numpy()
-        for b in range(B):
+        for b in range(w.B):
             assert (tok[b, :L[b] + 1] == tt[b, :L[b] + 1]).all()
             assert (dt[b, :L[b]] == tt[b, :L[b]]).all()
             assert L[b] == w.k or dt[b, L[b]] != tt[b, L[b]]
-    # sampled sequences, one by one, against the oracle (sequence id kept)
-    for b in sample:
-        sub = dict(target=inp["target"][b:b + 1], draft=inp["draft"][b:b + 1], seeds=inp["seeds"][b:b + 1],
-                   T=inp["T"], temps=None if inp.get("temps") is None else inp["temps"][b:b + 1],
-                   parent=inp.get("parent"))
-        sub_out = {k: v[b:b + 1] for k, v in out.items()}
-        check_verify(sub, sub_out, seq_ids=[b])
-    return L
+    flips = check_verify(inp, out)          # all B sequences, every row
+    return inp, out, flips
 
 
-def test_config3_full_size_sampled(ersd):
-    L = _full_size_sampled(ersd, "c3", sample=(0, 31, 63), sigma=1.0, T=1.0)
-    assert 0.05 < (L > 0).mean() < 1.0
-
-
-def test_config4_full_size_sampled(ersd):
-    _full_size_sampled(ersd, "c4", sample=(0, 31))
-
-
-def test_config5_full_size_sampled(ersd):
-    _full_size_sampled(ersd, "c5", sample=(0, 100, 255))
-
-
-def test_acceptance_tracks_the_closed_form_at_full_vocabulary(ersd):
-    """Config 2 over many calls: the number of accepted first positions falls within 4.5 sigma of
-    the sum of the rows' closed-form match probabilities (computed at full V by sorting on p/q)."""
-    w = wl.CONFIGS["c2"]
-    exp_sum, var_sum, got = 0.0, 0.0, 0
-    for call in range(10, 40):
-        inp = wl.make_inputs(w, call=call)
-        d = to_dev(inp)
-        out = ersd.verify(d["target"], d["draft"], d["seeds"], d["T"])
-        got += int((out["accept_len"] >= 1).sum().item())
-        p = torch.softmax(inp["target"][:, 0].double(), -1).numpy()
-        q = torch.softmax(inp["draft"][:, 0].double(), -1).numpy()
-        for b in range(w.B):
-            r = p[b] / q[b]
-            o = np.argsort(r)
-            ps, qs, rs = p[b][o], q[b][o], r[o]
-            tail_p = np.cumsum(ps[::-1])[::-1]                 # sum of p_j over r_j >= r_i
-            head_q = np.concatenate([[0.0], np.cumsum(qs)[:-1]])  # sum of q_j over r_j < r_i
-            m = float((1.0 / (tail_p / ps + head_q / qs)).sum())
+def test_config3_sweep_full_size(ersd):
+    """Config 3 as stated: all six (sigma, T) points at B=64, k=8, V=128256, every sequence against
+    the oracle; and over the sweep the accepted first positions within 4.5 sigma of the closed
+    form sum_i 1 / sum_j max(p_j/p_i, q_j/q_i) summed over the 384 first rows (Section 3)."""
+    exp_sum, var_sum, got, flips = 0.0, 0.0, 0, 0
+    rates = {}
+    for sigma, T in wl.C3_SWEEP:
+        inp, out, f = _full_size(ersd, "c3", sigma=sigma, T=T)
+        flips += f
+        acc1 = (out["accept_len"] >= 1).cpu().numpy()
+        got += int(acc1.sum())
+        rates[(sigma, T)] = float(out["accept_len"].float().mean().item())
+        p = torch.softmax(inp["target"][:, 0].double() / T, -1).cpu().numpy()
+        q = torch.softmax(inp["draft"][:, 0].double() / T, -1).cpu().numpy()
+        for b in range(p.shape[0]):
+            m = closed_form_match(p[b], q[b])
             exp_sum += m
             var_sum += m * (1 - m)
+    print("config 3 sweep: mean accepted length per point", rates, "near-tie rows taken the other way:", flips)
+    assert flips <= 1
     assert abs(got - exp_sum) < 4.5 * math.sqrt(var_sum), (got, exp_sum)
+    # a larger draft perturbation lowers acceptance (Section 3: the match rate falls with the distance of Q from P)
+    for T in (0.7, 1.0):
+        assert rates[(0.25, T)] > rates[(1.0, T)] > rates[(2.0, T)]
 
 
-# ------------------------------------------------------------------ edge cases
+def test_config4_tree_full_size(ersd):
+    _, out, flips = _full_size(ersd, "c4")
+    assert flips <= 1
+    assert out["tokens"].shape == (32, 5)
+
+
+def test_config5_full_size(ersd):
+    _, out, flips = _full_size(ersd, "c5")
+    print("config 5: near-tie rows taken the other way:", flips)
+    assert flips <= 1
+
+
 @pytest.mark.parametrize("V", [1, 2, 3, 5, 7, 8, 9, 31, 1023, 1024, 1025, 2047, 2048, 2049, 4100, 20000])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_small_and_ragged_vocabularies(ersd, V, dtype):
@@ -626,3 +665,121 @@ def test_host_buffer_entry(ersd):
     ref = oracle.verify(wl.as_numpy_logits(inp["target"]), wl.as_numpy_logits(inp["draft"]),
                         wl.seeds_as_u64(inp["seeds"]), T=inp["T"])
     assert (acc.numpy() == ref["accept_len"]).all()
+
+
+# ------------------------------------------------------------------ near-tie counter, streams
+@pytest.mark.parametrize("split", [0, 3])
+def test_near_tie_counter_counts_engineered_near_ties(ersd, split):
+    """opts->near_tie_count: rows whose two best keys are closer than 1e-5 are counted, others are
+    not.  Rows of equal logits, the runner-up's logit raised until its key sits 5e-6 (even rows) or
+    1e-3 (odd rows) above the leader's."""
+    import oracle
+    B, V, T = 12, 40000, 1.0
+    seeds = wl.make_seeds(77, 0, B)
+    flat = np.zeros((B, 1, V), dtype=np.float32)
+    tok2, key2 = oracle.race_sample(flat, wl.seeds_as_u64(seeds), T=T, c=2)
+    logits = torch.zeros(B, 1, V, dtype=torch.float32)
+    for b in range(B):
+        gap = 5e-6 if b % 2 == 0 else 1e-3
+        logits[b, 0, int(tok2[b, 0, 1])] = float((key2[b, 0, 1] - key2[b, 0, 0] - gap) * T)
+    ref_tok, ref_key = oracle.race_sample(logits.numpy(), wl.seeds_as_u64(seeds), T=T, c=1)
+    gaps = ref_key[:, 0, 1] - ref_key[:, 0, 0]
+    assert ((gaps < 1e-5) == (np.arange(B) % 2 == 0)).all()          # the construction holds in the oracle's arithmetic
+    near = torch.zeros(1, dtype=torch.int32, device="cuda")
+    tok = torch.empty(B, 1, 1, dtype=torch.int32, device="cuda")
+    key = torch.empty(B, 1, 1, dtype=torch.float32, device="cuda")
+    d, s = logits.cuda(), seeds.cuda()
+    ersd.ersd_race_sample(d, s, T, tok, ersd.make_opts(near_tie_count=near, out_key=key, split_v=split))
+    torch.cuda.synchronize()
+    assert near.item() == B // 2
+    check_sample(logits, seeds, T, tok, key)                          # either winner is right on the near-tie rows
+    assert (tok[1::2, 0, 0].cpu().numpy() == ref_tok[1::2, 0, 0]).all()
+    ersd.ersd_race_sample(d, s, T, tok, ersd.make_opts(near_tie_count=near, split_v=split))
+    torch.cuda.synchronize()
+    assert near.item() == B                                           # the call adds to the counter
+    # the counter asks for the streaming kernel: the cluster kernel keeps no runner-up
+    with pytest.raises(ersd.ErsdError) as e:
+        ersd.ersd_race_sample(d, s, T, tok, ersd.make_opts(near_tie_count=near, kernel_path=2))
+    assert e.value.status == -3
+
+
+def test_near_tie_counter_on_verification_and_trees(ersd):
+    """The same counter over sequence and tree verification: it equals the number of races whose
+    consecutive arrivals (first c + 1) the oracle sees closer than 1e-5 -- none on these inputs,
+    one per planted pair -- and asking for it changes no result."""
+    import oracle
+    near = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for name, scale in (("c5", dict(B=6)), ("c4", dict(B=2)), ("c2", {})):
+        w = wl.scaled(wl.CONFIGS[name], **scale)
+        inp = wl.make_inputs(w, call=3)
+        base = run_verify(ersd, inp)
+        d = to_dev(inp)
+        kw = {}
+        if d.get("temps") is not None:
+            kw = dict(temps=d["temps"], temp_strides=(d["temps"].stride(0), d["temps"].stride(1)))
+        tok, acc = torch.empty_like(base["tokens"]), torch.empty_like(base["accept_len"])
+        near.zero_()
+        if w.is_tree:
+            ersd.ersd_verify_tree(d["target"], d["draft"], d["parent"], d["seeds"], d["T"], tok, acc,
+                                  ersd.make_opts(near_tie_count=near, **kw))
+            ref = oracle.verify_tree(wl.as_numpy_logits(inp["target"]), wl.as_numpy_logits(inp["draft"]),
+                                     inp["parent"], wl.seeds_as_u64(inp["seeds"]), T=inp["T"])
+            _, _, nchild, _ = oracle.tree_shape(inp["parent"])
+            want = int(((ref["target_key"][..., 1] - ref["target_key"][..., 0]) < 1e-5).sum())
+            for n in range(len(nchild)):
+                if nchild[n]:
+                    g = np.diff(ref["arrival_key"][:, n, :nchild[n] + 1], axis=-1)
+                    want += int((g < 1e-5).any(axis=-1).sum())
+        else:
+            ersd.ersd_verify(d["target"], d["draft"], d["seeds"], d["T"], tok, acc,
+                             ersd.make_opts(near_tie_count=near, **kw))
+            temps = None if inp.get("temps") is None else inp["temps"].numpy()
+            ref = oracle.verify(wl.as_numpy_logits(inp["target"]), wl.as_numpy_logits(inp["draft"]),
+                                wl.seeds_as_u64(inp["seeds"]), T=inp["T"], temps=temps)
+            want = sum(int(((ref[k][..., 1] - ref[k][..., 0]) < 1e-5).sum()) for k in ("target_key", "draft_key"))
+        torch.cuda.synchronize()
+        assert near.item() == want, (name, near.item(), want)
+        assert (tok == base["tokens"]).all() and (acc == base["accept_len"]).all()
+
+
+def test_two_streams_with_their_own_workspaces(ersd):
+    """Calls that overlap on the GPU must not share a workspace: two streams, each with its own,
+    verify different batches at the same time; both results equal the oracle's.  A call on a side
+    stream that makes the library's private workspace grow is ordered correctly too."""
+    w = wl.scaled(wl.CONFIGS["c2"], B=48, V=20000)
+    inps = [wl.make_inputs(w, call=500 + i) for i in range(2)]
+    devs = [to_dev(i) for i in inps]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    nbytes = ersd.ersd_workspace_bytes(w.B, w.k + 1)
+    outs = []
+    torch.cuda.synchronize()
+    for rep in range(3):
+        outs = []
+        for d, st in zip(devs, streams):
+            ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+            with torch.cuda.stream(st):
+                ersd.ersd_workspace_init(ws, st)
+                o = dict(tokens=torch.empty(w.B, w.k + 1, dtype=torch.int32, device="cuda"),
+                         accept_len=torch.empty(w.B, dtype=torch.int32, device="cuda"),
+                         draft_tok=torch.empty(w.B, w.k, dtype=torch.int32, device="cuda"),
+                         draft_key=torch.empty(w.B, w.k, dtype=torch.float32, device="cuda"),
+                         target_tok=torch.empty(w.B, w.k + 1, dtype=torch.int32, device="cuda"),
+                         target_key=torch.empty(w.B, w.k + 1, dtype=torch.float32, device="cuda"))
+                ersd.ersd_verify(d["target"], d["draft"], d["seeds"], d["T"], o["tokens"], o["accept_len"],
+                                 ersd.make_opts(workspace=ws, out_draft_tok=o["draft_tok"], out_draft_key=o["draft_key"],
+                                                out_target_tok=o["target_tok"], out_target_key=o["target_key"]), st)
+            outs.append((o, ws))
+        for st in streams:
+            st.synchronize()
+        for inp, (o, _) in zip(inps, outs):
+            check_verify(inp, o)
+    # private workspace grown by a call on a side stream (700 x 9 rows: more than any call before it)
+    big = wl.Workload("grow", B=700, k=8, V=2100, dtype="bf16", sigma=0.7, T=1.0, config_id=49)
+    inp = wl.make_inputs(big, call=1)
+    d = to_dev(inp)
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        out = ersd.verify(d["target"], d["draft"], d["seeds"], d["T"], want_rows=True)
+    side.synchronize()
+    check_verify(inp, out)
