@@ -210,6 +210,61 @@ int ersd_verify_tokens(const void* target_logits, const int32_t* draft_tokens, e
                        int32_t* out_accept_len, const ersd_opts* opts, void* cuda_stream);
 
 /*
+ * Greedy speculative decoding (GSD) on the same logits -- the verifier the paper
+ * compares ERSD with (Algorithm 1, Section 2, applied position by position:
+ * drafted tokens are verified in order until the first rejection).  For every
+ * sequence b and position j < k, in order:
+ *   x = draft_tokens[b, j], a sample of softmax(draft row j / T) made earlier
+ *       (any sampler; ersd_race_sample on the draft rows is one);
+ *   accept iff P_j(x) / Q_j(x) > u, with P_j, Q_j the softmax of target / draft
+ *       row j and u ~ Uniform(0, 1);
+ *   on the first rejection emit a sample of max(P_j - Q_j, 0) / sum and stop;
+ *   after k acceptances emit a sample of softmax(target row k / T).
+ * Randomness (the paper names none): u is word 0 of Philox4x32-10 under the
+ * sequence's key with counter (0, position, sequence id, 1), u = (x + 1/2) 2^-32;
+ * the token that ends the call is the winner of an exponential race over the
+ * residual (or target) law, argmin_i e_i / w_i, with e_i from counter
+ * (i >> 2, position, sequence id, 2) -- both independent of the drafting races
+ * (last counter word 0), as Algorithm 1 requires.  All arithmetic is double
+ * precision; the call is four small launches, not the single streaming launch
+ * of ersd_verify.
+ *   target_logits device [B, k+1, V]   draft_logits device [B, k, V]
+ *   draft_tokens  device [B, k] int32  out_tokens device [B, k+1] int32 (-1 padded)
+ *   out_accept_len device [B] int32
+ * opts: ld_*, temps (every temperature must be > 0), seq_ids, pos_offsets,
+ * workspace (ersd_workspace_bytes(B, k + 1) bytes, as for ersd_verify; left zeroed).
+ * Errors as for ersd_verify; T <= 0 is ERSD_EINVAL (the test needs a softmax).
+ */
+int ersd_gsd_verify(const void* target_logits, const void* draft_logits, const int32_t* draft_tokens,
+                    ersd_dtype dt, const uint64_t* seeds, int B, int k, int V, float T, int32_t* out_tokens,
+                    int32_t* out_accept_len, const ersd_opts* opts, void* cuda_stream);
+
+/*
+ * Tree GSD (Algorithm 4, Appendix A; the algorithm is printed with the tested
+ * token's child index missing and an empty loop -- the reading taken is Section
+ * 2's text: recursive batch selection).  Tree layout as for ersd_verify_tree
+ * (`parent` a HOST array).  draft_tokens[b, n] is the token drafted at node n
+ * (entry 0 unused); siblings must have been drafted WITHOUT replacement from
+ * their parent's draft row (the first arrivals of ersd_race_sample with top_c
+ * are).  Walk from the root: the current node's children are tried in order;
+ * child of rank i is accepted iff P_t(x) / Q_d(x) > u(node, i), where every
+ * rejection replaces P_t by max(P_t - Q_d, 0) / sum and removes the rejected
+ * token from Q_d (renormalised); an accepted child becomes the current node with
+ * its own rows; when no child is accepted, or at a leaf, a sample of the current
+ * P_t is emitted and the call ends.  u(node, i): counter (i, node, sequence id, 1);
+ * the final race: counter (token >> 2, node, sequence id, 2).
+ *   target_logits, draft_logits device [B, N+1, V] (draft rows of leaves never read)
+ *   draft_tokens device [B, N+1] int32   out_tokens device [B, D+1] int32 (-1 padded)
+ *   out_accept_len device [B] int32      opts->out_path as for ersd_verify_tree
+ * One thread block walks one sequence, in double precision: a comparison path,
+ * not a throughput path.
+ */
+int ersd_gsd_verify_tree(const void* target_logits, const void* draft_logits, const int32_t* draft_tokens,
+                         ersd_dtype dt, const int32_t* parent, const uint64_t* seeds, int B, int N, int V,
+                         float T, int32_t* out_tokens, int32_t* out_accept_len, const ersd_opts* opts,
+                         void* cuda_stream);
+
+/*
  * ersd_verify for callers that must not allocate device memory.  (The paper has
  * no counterpart; this is a deployment variant of ersd_verify and computes
  * exactly the same outputs from the same arguments.)

@@ -22,7 +22,7 @@ ERSD_MAX_TOP_C, ERSD_MAX_ROWS, ERSD_MAX_SPLIT = 32, 256, 32
 ERSD_NOALLOC_MAX_ROWS = 1024
 ERSD_ENOALLOC_LIMIT = -6
 
-EXPORTS = ("ersd_race_sample", "ersd_verify", "ersd_verify_tokens", "ersd_verify_noalloc", "ersd_verify_tree", "ersd_tree_depth", "ersd_optimal_tree",
+EXPORTS = ("ersd_race_sample", "ersd_verify", "ersd_verify_tokens", "ersd_verify_noalloc", "ersd_verify_tree", "ersd_gsd_verify", "ersd_gsd_verify_tree", "ersd_tree_depth", "ersd_optimal_tree",
            "ersd_row_keys", "ersd_workspace_bytes", "ersd_workspace_init", "ersd_status_string",
            "ersd_last_cuda_error", "ersd_version")
 
@@ -70,6 +70,9 @@ def lib():
         L.ersd_verify_tokens.argtypes = L.ersd_verify.argtypes
         L.ersd_verify_tree.argtypes = [vp, vp, i, C.POINTER(C.c_int32), vp, i, i, i, f, vp, vp,
                                        C.POINTER(ErsdOpts), vp]
+        L.ersd_gsd_verify.argtypes = [vp, vp, vp, i, vp, i, i, i, f, vp, vp, C.POINTER(ErsdOpts), vp]
+        L.ersd_gsd_verify_tree.argtypes = [vp, vp, vp, i, C.POINTER(C.c_int32), vp, i, i, i, f, vp, vp,
+                                           C.POINTER(ErsdOpts), vp]
         L.ersd_tree_depth.argtypes = [C.POINTER(C.c_int32), i]
         L.ersd_optimal_tree.argtypes = [C.POINTER(C.c_double), i, i, C.POINTER(C.c_int32), C.POINTER(C.c_double)]
         L.ersd_optimal_tree.restype = i
@@ -80,6 +83,7 @@ def lib():
         L.ersd_status_string.argtypes = [i]
         L.ersd_status_string.restype = C.c_char_p
         for name in ("ersd_race_sample", "ersd_verify", "ersd_verify_tokens", "ersd_verify_noalloc", "ersd_verify_tree", "ersd_tree_depth",
+                     "ersd_gsd_verify", "ersd_gsd_verify_tree",
                      "ersd_row_keys", "ersd_workspace_init", "ersd_last_cuda_error", "ersd_version"):
             getattr(L, name).restype = i
         _lib = L
@@ -237,6 +241,50 @@ def ersd_verify_tokens(target_logits: torch.Tensor, draft_tokens: Optional[torch
                                     _ptr(seeds), B, rows - 1, V, float(T), _ptr(out_tokens),
                                     _ptr(out_accept_len), C.byref(opts) if opts is not None else None,
                                     _stream(stream)), "ersd_verify_tokens")
+
+
+def ersd_gsd_verify(target_logits: torch.Tensor, draft_logits: Optional[torch.Tensor],
+                    draft_tokens: Optional[torch.Tensor], seeds: torch.Tensor, T: float, out_tokens: torch.Tensor,
+                    out_accept_len: torch.Tensor, opts: Optional[ErsdOpts] = None, stream=None,
+                    V: Optional[int] = None) -> None:
+    """Greedy speculative decoding (Algorithm 1 position by position) on the same logits.
+    target [B, k+1, V], draft [B, k, V], draft_tokens int32 [B, k]; out_tokens int32 [B, k+1]."""
+    _dev(target_logits, None, "target_logits")
+    B, rows, V = _sizes(target_logits, V)
+    if draft_logits is not None:
+        _dev(draft_logits, target_logits.dtype, "draft_logits")
+    if draft_tokens is not None:
+        _dev(draft_tokens, torch.int32, "draft_tokens")
+    _dev(seeds, torch.int64, "seeds")
+    _dev(out_tokens, torch.int32, "out_tokens")
+    _dev(out_accept_len, torch.int32, "out_accept_len")
+    _check(lib().ersd_gsd_verify(_ptr(target_logits), _ptr(draft_logits), _ptr(draft_tokens),
+                                 _dtype_code(target_logits), _ptr(seeds), B, rows - 1, V, float(T),
+                                 _ptr(out_tokens), _ptr(out_accept_len),
+                                 C.byref(opts) if opts is not None else None, _stream(stream)), "ersd_gsd_verify")
+
+
+def ersd_gsd_verify_tree(target_logits: torch.Tensor, draft_logits: Optional[torch.Tensor],
+                         draft_tokens: Optional[torch.Tensor], parent: Sequence[int], seeds: torch.Tensor,
+                         T: float, out_tokens: torch.Tensor, out_accept_len: torch.Tensor,
+                         opts: Optional[ErsdOpts] = None, stream=None, V: Optional[int] = None) -> None:
+    """Tree GSD (Algorithm 4).  target, draft [B, N+1, V]; draft_tokens int32 [B, N+1] (entry 0
+    unused); parent: host list [N+1]; out_tokens int32 [B, D+1]."""
+    _dev(target_logits, None, "target_logits")
+    B, rows, V = _sizes(target_logits, V)
+    if draft_logits is not None:
+        _dev(draft_logits, target_logits.dtype, "draft_logits")
+    if draft_tokens is not None:
+        _dev(draft_tokens, torch.int32, "draft_tokens")
+    _dev(seeds, torch.int64, "seeds")
+    _dev(out_tokens, torch.int32, "out_tokens")
+    _dev(out_accept_len, torch.int32, "out_accept_len")
+    arr = (C.c_int32 * len(parent))(*[int(x) for x in parent])
+    _check(lib().ersd_gsd_verify_tree(_ptr(target_logits), _ptr(draft_logits), _ptr(draft_tokens),
+                                      _dtype_code(target_logits), arr, _ptr(seeds), B, rows - 1, V, float(T),
+                                      _ptr(out_tokens), _ptr(out_accept_len),
+                                      C.byref(opts) if opts is not None else None, _stream(stream)),
+           "ersd_gsd_verify_tree")
 
 
 def ersd_verify_noalloc(target_logits: torch.Tensor, draft_logits: Optional[torch.Tensor],

@@ -641,6 +641,58 @@ static int noalloc_scratch(void** out) {
   return ERSD_OK;
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Greedy speculative decoding (the paper's comparison verifier): kernels and launch logic.
+// ---------------------------------------------------------------------------------------------
+#include "ersd_gsd.inc"
+
+// Scratch of a sequence-GSD call, carved from the front of the workspace: softmax statistics
+// [B, 2k+1, 2] doubles, partial winners [B, S] (double, int), first rejections [B].
+static size_t gsd_scratch_bytes(int64_t B, int64_t k, int64_t S) {
+  return (size_t)(B * ((2 * k + 1) * 16 + S * 16 + 8));
+}
+
+static int gsd_check(const void* target, const void* draft, const int32_t* draft_tok, int dt,
+                     const uint64_t* seeds, int B, int rows, int V, float T, const void* out_tokens,
+                     const void* out_accept_len, bool need_draft) {
+  int st = check_common(target, dt, seeds, B, rows, V, T);
+  if (st != ERSD_OK) return st;
+  if (!(T > 0.0f)) return ERSD_EINVAL;  // the ratio test needs softmax(z / T)
+  if (!out_tokens || !out_accept_len) return ERSD_EINVAL;
+  if (need_draft) {
+    if (!draft || !draft_tok) return ERSD_EINVAL;
+    if (((uintptr_t)draft & (elem_size(dt) - 1)) != 0 || ((uintptr_t)draft_tok & 3) != 0) return ERSD_EALIGN;
+  }
+  return ERSD_OK;
+}
+
+static void gsd_fill(GsdParams& g, const ersd_opts& o, const void* target, const void* draft,
+                     const int32_t* draft_tok, const uint64_t* seeds, int B, int k, int V, float T,
+                     int rows_t, int rows_d, int32_t* out_tokens, int32_t* out_accept_len) {
+  memset(&g, 0, sizeof g);
+  g.target = target;
+  g.draft = draft;
+  g.draft_tok = draft_tok;
+  g.seeds = seeds;
+  g.seq_ids = o.seq_ids;
+  g.pos_offsets = o.pos_offsets;
+  g.temps = o.temps;
+  g.ts_b = o.temp_stride_b;
+  g.ts_r = o.temp_stride_r;
+  g.ld_t = o.ld_target ? o.ld_target : V;
+  g.ld_d = o.ld_draft ? o.ld_draft : V;
+  g.T = T;
+  g.B = B;
+  g.k = k;
+  g.V = V;
+  g.rows_t = rows_t;
+  g.rows_d = rows_d;
+  g.out_tokens = out_tokens;
+  g.out_accept_len = out_accept_len;
+  g.out_path = o.out_path;
+}
+
 }  // namespace ersd
 
 using namespace ersd;
@@ -794,6 +846,84 @@ int ersd_verify_noalloc(const void* target_logits, const void* draft_logits, ers
   if (e != cudaSuccess) return cuda_fail(e);
   return verify_sequence(target_logits, draft_logits, dt, seeds, B, k, V, T, out_tokens, out_accept_len, &o,
                          cuda_stream, false);
+}
+
+
+int ersd_gsd_verify(const void* target_logits, const void* draft_logits, const int32_t* draft_tokens,
+                    ersd_dtype dt, const uint64_t* seeds, int B, int k, int V, float T, int32_t* out_tokens,
+                    int32_t* out_accept_len, const ersd_opts* opts, void* cuda_stream) {
+  if (k < 0) return ERSD_EINVAL;
+  if (k + 1 > ERSD_MAX_ROWS) return ERSD_EUNSUPPORTED;
+  int st = gsd_check(target_logits, draft_logits, draft_tokens, dt, seeds, B, k + 1, V, T, out_tokens,
+                     out_accept_len, k > 0);
+  if (st != ERSD_OK) return st;
+  const ersd_opts o = read_opts(opts);
+  GsdParams g;
+  gsd_fill(g, o, target_logits, draft_logits, draft_tokens, seeds, B, k, V, T, k + 1, k, out_tokens,
+           out_accept_len);
+  if (g.ld_t < V || g.ld_d < V) return ERSD_EINVAL;
+  // slices of the final race: about two blocks per multiprocessor in all, at least 4096 tokens each
+  int S = (2 * sm_count() + B - 1) / B;
+  if (S > (V + 4095) / 4096) S = (V + 4095) / 4096;
+  if (S > 64) S = 64;
+  if (S < 1) S = 1;
+  g.S = S;
+  const size_t need = gsd_scratch_bytes(B, k, S);  // (never more than ersd_workspace_bytes(B, k + 1))
+  void* ws = nullptr;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  st = get_workspace(o, workspace_bytes(B, k + 1), &ws, stream);
+  if (st != ERSD_OK) return st;
+  char* w = (char*)ws;
+  g.stats = (double*)w;
+  w += (size_t)B * (2 * k + 1) * 16;
+  g.part_t = (double*)w;
+  w += (size_t)B * S * 8;
+  g.part_i = (int*)w;
+  w += (size_t)B * S * 4;
+  g.jstar = (int*)w;
+  const dim3 rows_grid((unsigned)(2 * k + 1), (unsigned)B), race_grid((unsigned)S, (unsigned)B);
+  const unsigned seq_blocks = (unsigned)((B + 127) / 128);
+  if (dt == ERSD_BF16) {
+    gsd_stats_kernel<ERSD_BF16><<<rows_grid, kGsdThreads, 0, stream>>>(g);
+    gsd_scan_kernel<ERSD_BF16><<<seq_blocks, 128, 0, stream>>>(g);
+    gsd_race_kernel<ERSD_BF16><<<race_grid, kGsdThreads, 0, stream>>>(g);
+  } else {
+    gsd_stats_kernel<ERSD_F32><<<rows_grid, kGsdThreads, 0, stream>>>(g);
+    gsd_scan_kernel<ERSD_F32><<<seq_blocks, 128, 0, stream>>>(g);
+    gsd_race_kernel<ERSD_F32><<<race_grid, kGsdThreads, 0, stream>>>(g);
+  }
+  gsd_finish_kernel<<<seq_blocks, 128, 0, stream>>>(g);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  // the workspace's resting state is all zero (the race kernels' arrival counters count on it)
+  e = cudaMemsetAsync(ws, 0, need, stream);
+  return e == cudaSuccess ? ERSD_OK : cuda_fail(e);
+}
+
+int ersd_gsd_verify_tree(const void* target_logits, const void* draft_logits, const int32_t* draft_tokens,
+                         ersd_dtype dt, const int32_t* parent, const uint64_t* seeds, int B, int N, int V,
+                         float T, int32_t* out_tokens, int32_t* out_accept_len, const ersd_opts* opts,
+                         void* cuda_stream) {
+  if (N < 0 || !parent) return ERSD_EINVAL;
+  if (N + 1 > ERSD_MAX_ROWS) return ERSD_EUNSUPPORTED;
+  int st = gsd_check(target_logits, draft_logits, draft_tokens, dt, seeds, B, N + 1, V, T, out_tokens,
+                     out_accept_len, N > 0);
+  if (st != ERSD_OK) return st;
+  TreeDesc tree;
+  int D = 0, cmax = 1;
+  st = build_tree(parent, N, &tree, &D, &cmax);
+  if (st != ERSD_OK) return st;
+  const ersd_opts o = read_opts(opts);
+  GsdParams g;
+  gsd_fill(g, o, target_logits, draft_logits, draft_tokens, seeds, B, N, V, T, N + 1, N + 1, out_tokens,
+           out_accept_len);
+  if (g.ld_t < V || g.ld_d < V) return ERSD_EINVAL;
+  g.depth = D;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  if (dt == ERSD_BF16) gsd_tree_kernel<ERSD_BF16><<<(unsigned)B, kGsdTreeThreads, 0, stream>>>(g, tree);
+  else gsd_tree_kernel<ERSD_F32><<<(unsigned)B, kGsdTreeThreads, 0, stream>>>(g, tree);
+  const cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? ERSD_OK : cuda_fail(e);
 }
 
 int ersd_tree_depth(const int32_t* parent, int N) {
