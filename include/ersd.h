@@ -322,6 +322,25 @@ int ersd_verify_noalloc(const void* target_logits, const void* draft_logits, ers
 int ersd_optimal_tree(const double* accept, int max_children, int k, int32_t* parent_out,
                       double* expected_tokens);
 
+/*
+ * Empirical acceptance profile for ersd_optimal_tree (Section 5 of the paper: the
+ * acceptance probability function R is estimated from observed acceptances and
+ * treated as a 0-th order Markov source).  HOST function, no GPU work.
+ *   paths   HOST [B, D+1]: accepted node ids per sequence, -1 padded -- what
+ *           opts->out_path of ersd_verify_tree (or ersd_gsd_verify_tree) returns,
+ *           copied to the host; D = ersd_tree_depth(parent, N)
+ *   parent  HOST [N+1]: the draft tree those calls verified
+ *   accept  HOST [max_children] out: accept[r] = (times a child of rank r was the
+ *           accepted one) / (times a node with a child of rank r was verified);
+ *           0 where never tried; capped so that it never rises with r, the form
+ *           ersd_optimal_tree takes
+ *   trials  HOST [max_children] out, nullable: the denominators
+ * Errors: ERSD_EINVAL (null pointers, malformed parent array, a path that is not
+ * a root path of the tree); ERSD_EUNSUPPORTED for N + 1 > ERSD_MAX_ROWS.
+ */
+int ersd_acceptance_profile(const int32_t* paths, const int32_t* parent, int B, int N, int max_children,
+                            double* accept, int64_t* trials);
+
 /* Depth (longest root-to-leaf edge count) of a HOST parent array, or -1 if it is malformed. */
 int ersd_tree_depth(const int32_t* parent, int N);
 

@@ -92,3 +92,27 @@ def parent_array(paths) -> List[int]:
     order = [()] + sorted(tuple(p) for p in paths)
     index = {p: n for n, p in enumerate(order)}
     return [-1] + [index[p[:-1]] for p in order[1:]]
+
+
+def acceptance_profile(paths, parent: Sequence[int], max_children: int):
+    """Empirical per-rank acceptance (Section 5: R estimated from observed acceptances as a 0-th
+    order Markov source).  `paths`: per sequence the accepted node ids, root first (-1 padding
+    allowed).  A node on a path was verified: each of its children is one trial of its rank; the
+    next node on the path is the child that was accepted.  Returns (accept, trials) per rank, with
+    accept[r] = hits[r] / trials[r] (0 where never tried), uncapped."""
+    n = len(parent)
+    kids = [[] for _ in range(n)]
+    for m in range(1, n):
+        kids[parent[m]].append(m)
+    hits = [0] * max_children
+    trials = [0] * max_children
+    for path in paths:
+        path = [int(v) for v in path if int(v) >= 0]
+        for d, node in enumerate(path):
+            for r in range(min(len(kids[node]), max_children)):
+                trials[r] += 1
+            if d + 1 < len(path):
+                r = kids[node].index(path[d + 1])
+                if r < max_children:
+                    hits[r] += 1
+    return [hits[r] / trials[r] if trials[r] else 0.0 for r in range(max_children)], trials

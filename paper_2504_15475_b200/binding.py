@@ -23,7 +23,7 @@ ERSD_NOALLOC_MAX_ROWS = 1024
 ERSD_ENOALLOC_LIMIT = -6
 
 EXPORTS = ("ersd_race_sample", "ersd_verify", "ersd_verify_tokens", "ersd_verify_noalloc", "ersd_verify_tree", "ersd_gsd_verify", "ersd_gsd_verify_tree", "ersd_tree_depth", "ersd_optimal_tree",
-           "ersd_row_keys", "ersd_workspace_bytes", "ersd_workspace_init", "ersd_status_string",
+           "ersd_acceptance_profile", "ersd_row_keys", "ersd_workspace_bytes", "ersd_workspace_init", "ersd_status_string",
            "ersd_last_cuda_error", "ersd_version")
 
 
@@ -76,6 +76,9 @@ def lib():
         L.ersd_tree_depth.argtypes = [C.POINTER(C.c_int32), i]
         L.ersd_optimal_tree.argtypes = [C.POINTER(C.c_double), i, i, C.POINTER(C.c_int32), C.POINTER(C.c_double)]
         L.ersd_optimal_tree.restype = i
+        L.ersd_acceptance_profile.argtypes = [C.POINTER(C.c_int32), C.POINTER(C.c_int32), i, i, i,
+                                              C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+        L.ersd_acceptance_profile.restype = i
         L.ersd_row_keys.argtypes = [vp, i, i, f, C.c_uint64, C.c_uint32, C.c_uint32, i, vp, vp]
         L.ersd_workspace_bytes.argtypes = [i, i]
         L.ersd_workspace_bytes.restype = C.c_size_t
@@ -192,6 +195,20 @@ def ersd_optimal_tree(accept: Sequence[float], k: int):
     expected = C.c_double(0.0)
     _check(lib().ersd_optimal_tree(a, len(accept), int(k), parent, C.byref(expected)), "ersd_optimal_tree")
     return list(parent), float(expected.value)
+
+
+def ersd_acceptance_profile(paths, parent: Sequence[int], max_children: int):
+    """(accept [max_children], trials [max_children]) from the accepted paths ([B, D+1] node ids,
+    -1 padded: opts.out_path of a tree verification, any device) over the draft tree `parent`:
+    the empirical per-rank acceptance probabilities that ersd_optimal_tree takes (host function)."""
+    pt = torch.as_tensor(paths).detach().to("cpu", torch.int32).contiguous()
+    B = int(pt.shape[0])
+    par = (C.c_int32 * len(parent))(*[int(x) for x in parent])
+    acc = (C.c_double * max_children)()
+    tri = (C.c_int64 * max_children)()
+    _check(lib().ersd_acceptance_profile(C.cast(pt.data_ptr(), C.POINTER(C.c_int32)), par, B, len(parent) - 1,
+                                         int(max_children), acc, tri), "ersd_acceptance_profile")
+    return list(acc), list(tri)
 
 
 def ersd_race_sample(logits: torch.Tensor, seeds: torch.Tensor, T: float, out_tok: torch.Tensor,

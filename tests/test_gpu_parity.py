@@ -783,3 +783,34 @@ def test_two_streams_with_their_own_workspaces(ersd):
         out = ersd.verify(d["target"], d["draft"], d["seeds"], d["T"], want_rows=True)
     side.synchronize()
     check_verify(inp, out)
+
+
+def test_tree_built_from_measured_acceptance(ersd):
+    """Section 5's loop closed on synthetic rows: batch drafting (a star of 8) is verified, the
+    accepted paths give the empirical per-rank acceptance (0-th order R), Algorithm 3 builds the
+    16-token tree from it, and that tree, verified on fresh rows of the same recipe, accepts about
+    as many tokens as the model predicts and not fewer than the fixed 4 x 4 tree."""
+    V, B = 8192, 384
+    star = list(wl.star_parent(8))
+    w = wl.Workload("measure", B=B, k=8, V=V, dtype="bf16", sigma=1.0, T=1.0, config_id=51, parent=tuple(star))
+    inp = wl.make_inputs(w, call=0)
+    out = run_verify(ersd, inp)
+    check_verify(inp, out)
+    accept, trials = ersd.ersd_acceptance_profile(out["path"], star, 8)
+    assert trials[0] == B and all(accept[r] >= accept[r + 1] for r in range(7)) and 0.2 < accept[0] < 0.9
+    parent16, expected = ersd.ersd_optimal_tree(accept, 16)
+    means = {}
+    for name, parent in (("measured", parent16), ("4x4", list(wl.TREE_4x4))):
+        wt = wl.Workload(name, B=B, k=16, V=V, dtype="bf16", sigma=1.0, T=1.0, config_id=52, parent=tuple(parent))
+        it = wl.make_inputs(wt, call=1)
+        ot = run_verify(ersd, it)
+        check_verify(it, ot)
+        acc = ot["accept_len"].float()
+        means[name] = (acc.mean().item(), acc.std().item() / B ** 0.5)
+    m_opt, se_opt = means["measured"]
+    m_44, se_44 = means["4x4"]
+    print("accept profile", [round(a, 3) for a in accept], "predicted", round(expected, 3), "measured", means)
+    assert m_opt >= m_44 - 3 * (se_opt + se_44)
+    # every node's rows are independent draws of one recipe, so the 0-th order model holds and its
+    # prediction (from a profile that itself carries sampling noise) is met within a few standard errors
+    assert abs(m_opt - expected) < 5 * se_opt + 0.12
