@@ -33,7 +33,7 @@ if ROOT not in sys.path:
 # profiles/: dram bytes (read + write) per algorithmic byte of one launch, and the library version
 # the counters were taken at
 DRAM_BYTES_PER_ALGORITHMIC_BYTE = 1.024
-TRAFFIC_AT_VERSION = 108  # (version 108 changed the cluster kernel only: the counters of version 107 stand)
+TRAFFIC_AT_VERSION = 108  # (the counters were taken at this library version; another version reports traffic null)
 SM_COUNT = 148
 
 METRIC = "race-verified logit rows/s at V=128256 bf16 (B*(k+1) rows)"
@@ -106,6 +106,8 @@ def algorithmic_bytes(w, inp, entry="verify"):
     """Bytes one verify launch must read: every target row, every draft row that has children
     (token-given verification reads target rows only)."""
     es = inp["target"].element_size()
+    if entry == "gsd":
+        return (w.B * (w.rows_target + w.k) + 2 * w.B) * w.V * es
     if entry == "tokens":
         rows = w.B * w.rows_target
     elif w.is_tree:
@@ -189,6 +191,21 @@ def run_reference(args, w):
         "gpu_launches": 0}))
 
 
+L2_BYTES = 126e6
+
+
+def l2_note(bytes_per_launch, n_sets):
+    """How the timed launches relate to the L2: what the timing rules ask a bench line to say."""
+    mb = bytes_per_launch / 1e6
+    if bytes_per_launch > L2_BYTES:
+        return "inputs larger than L2 (%.0f MB per launch); %d input sets rotated" % (mb, n_sets)
+    if bytes_per_launch * n_sets > L2_BYTES:
+        return ("one input set (%.1f MB) fits the L2, the %d sets rotated between launches together do not"
+                % (mb, n_sets))
+    return ("inputs fit the L2 (%.2f MB per launch, %d sets): a latency figure, not an HBM one; "
+            "pass --sets N for more sets than the L2 holds" % (mb, n_sets))
+
+
 def workload_config(w, l2_note):
     return {"workload": "%s: B=%d k=%d V=%d %s %s" % (w.name, w.B, w.k, w.V, w.dtype,
                                                      "tree" if w.is_tree else "sequence"),
@@ -202,9 +219,10 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="c5")
-    ap.add_argument("--entry", default="verify", choices=["verify", "tokens"],
+    ap.add_argument("--entry", default="verify", choices=["verify", "tokens", "gsd"],
                     help="verify: ersd_verify / ersd_verify_tree (the headline path); tokens: "
-                         "ersd_verify_tokens on tokens drafted before the timed region")
+                         "ersd_verify_tokens on tokens drafted before the timed region; gsd: the "
+                         "comparison verifier ersd_gsd_verify (Algorithm 1) on tokens drafted before it")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sets", type=int, default=3, help="distinct input sets rotated between launches")
     ap.add_argument("--e2e-steps", type=int, default=4)
@@ -259,9 +277,9 @@ def main():
     all_opts = [opts_for(inp) for inp in sets]
 
     drafted = None
-    if args.entry == "tokens":
+    if args.entry in ("tokens", "gsd"):
         if w.is_tree:
-            raise SystemExit("--entry tokens takes a sequence workload")
+            raise SystemExit("--entry %s takes a sequence workload" % args.entry)
         drafted = []
         for inp, o in zip(sets, all_opts):     # drafting happens before the timed region
             d = torch.empty(w.B, w.k, 1, dtype=torch.int32, device="cuda")
@@ -276,7 +294,10 @@ def main():
 
     def step(i):
         inp = sets[i % len(sets)]
-        if drafted is not None:
+        if drafted is not None and args.entry == "gsd":
+            binding.ersd_gsd_verify(inp["target"], inp["draft"], drafted[i % len(sets)], inp["seeds"], inp["T"],
+                                    tokens, accept, all_opts[i % len(sets)], stream)
+        elif drafted is not None:
             binding.ersd_verify_tokens(inp["target"], drafted[i % len(sets)], inp["seeds"], inp["T"], tokens,
                                        accept, all_opts[i % len(sets)], stream)
         elif w.is_tree:
@@ -312,6 +333,7 @@ def main():
     clocks = sampler.stop(t_wall0, t_wall1)
     rows_per_step = w.B * w.rows_target
     value, ms_step = replicas.whole_job_rate(rows_per_step, args.steps, ev0.elapsed_time(ev1), dist, "cuda")
+    launched = "ersd_gsd_verify: statistics, scan, race and merge kernels" if args.entry == "gsd" else binding.ersd_last_launch()
     mean_accept = float(accept.float().mean().item())
 
     # ---- roofline of the one kernel a step launches
@@ -330,10 +352,10 @@ def main():
     t_hbm_ms = alg_bytes / (peak * 1e9) * 1e3
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": traffic, "peak_kind": peak_kind + " copy bandwidth",
-                "algorithmic_bytes_per_launch": alg_bytes, "kernel": "ersd_race_kernel<bf16>",
+                "algorithmic_bytes_per_launch": alg_bytes, "kernel": launched,
                 "kernel_ms": ms_step, "t_hbm_ms": t_hbm_ms, "t_int_ms": t_alu_ms,
                 "note": "t_int_ms: Philox integer work alone at the nominal 64 int lanes/clk/SM"}
-    if t_alu_ms > t_hbm_ms:
+    if t_alu_ms > t_hbm_ms and args.entry != "gsd":
         # fewer bytes per index than integer work (target rows only): the integer path is the roof
         int_ops = n_index * 9.25
         peak_ops = 64.0 * SM_COUNT * (clocks["sm_max_mhz"] or 1965.0) * 1e6 / 1e9
@@ -386,10 +408,11 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32 screen + f64 decision, u32 Philox", "data": "synthetic",
-            "config": dict(workload_config(w, "inputs larger than L2; %d input sets rotated" % len(sets)),
-                           entry="ersd_verify_tokens" if args.entry == "tokens" else
-                           ("ersd_verify_tree" if w.is_tree else "ersd_verify")),
-            "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps, "roofline": roofline,
+            "config": dict(workload_config(w, l2_note(alg_bytes, len(sets))),
+                           entry={"tokens": "ersd_verify_tokens", "gsd": "ersd_gsd_verify"}.get(
+                               args.entry, "ersd_verify_tree" if w.is_tree else "ersd_verify")),
+            "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * (4 if args.entry == "gsd" else 1),
+            "roofline": roofline,
             "cpu_baseline": cpu, "parity_on_cpu_sample": parity, "mean_accept_len": mean_accept}))
     if dist is not None:
         dist.destroy_process_group()

@@ -364,6 +364,9 @@ int ersd_workspace_init(void* workspace, size_t bytes, void* cuda_stream);
 
 const char* ersd_status_string(int status);
 int ersd_last_cuda_error(void); /* cudaError_t of the last failing runtime call on this thread */
+/* Which kernel this thread's last ersd_race_sample / ersd_verify* call launched and in what shape
+   (a short text for logs and benchmarks; "" before the first launch).  Diagnostic only. */
+const char* ersd_last_launch(void);
 int ersd_version(void);
 
 #ifdef __cplusplus

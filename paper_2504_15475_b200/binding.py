@@ -24,7 +24,7 @@ ERSD_ENOALLOC_LIMIT = -6
 
 EXPORTS = ("ersd_race_sample", "ersd_verify", "ersd_verify_tokens", "ersd_verify_noalloc", "ersd_verify_tree", "ersd_gsd_verify", "ersd_gsd_verify_tree", "ersd_tree_depth", "ersd_optimal_tree",
            "ersd_acceptance_profile", "ersd_row_keys", "ersd_workspace_bytes", "ersd_workspace_init", "ersd_status_string",
-           "ersd_last_cuda_error", "ersd_version")
+           "ersd_last_cuda_error", "ersd_last_launch", "ersd_version")
 
 
 class ErsdOpts(C.Structure):
@@ -85,6 +85,7 @@ def lib():
         L.ersd_workspace_init.argtypes = [vp, C.c_size_t, vp]
         L.ersd_status_string.argtypes = [i]
         L.ersd_status_string.restype = C.c_char_p
+        L.ersd_last_launch.restype = C.c_char_p
         for name in ("ersd_race_sample", "ersd_verify", "ersd_verify_tokens", "ersd_verify_noalloc", "ersd_verify_tree", "ersd_tree_depth",
                      "ersd_gsd_verify", "ersd_gsd_verify_tree",
                      "ersd_row_keys", "ersd_workspace_init", "ersd_last_cuda_error", "ersd_version"):
@@ -167,6 +168,11 @@ def make_opts(*, top_c: int = 0, split_v: int = 0, block_threads: int = 0, ld_ta
     if near_tie_count is not None:  # int32 tensor of one element that the call adds to
         o.near_tie_count = _dev(near_tie_count, torch.int32, "near_tie_count").data_ptr()
     return o
+
+
+def ersd_last_launch() -> str:
+    """Which kernel the last call of this thread launched, and in what shape."""
+    return lib().ersd_last_launch().decode()
 
 
 def ersd_version() -> int:

@@ -12,6 +12,7 @@
 // (sequence scan or tree walk) in the same launch.
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdio.h>
 #include <string.h>
 
 #include <mutex>
@@ -144,6 +145,7 @@ __global__ void ersd_row_keys_kernel(const void* row, int V, float T, uint64_t s
 // host side
 // ---------------------------------------------------------------------------------------------
 static thread_local int g_last_cuda_error = 0;
+static thread_local char g_last_launch[160] = "";  // ersd_last_launch(): what this thread's last call launched
 
 static int cuda_fail(cudaError_t e) {
   g_last_cuda_error = (int)e;
@@ -362,6 +364,8 @@ static int launch(const Params& p, const TreeDesc& tree, int dt, bool many, cuda
   const dim3 grid((unsigned)p.B, (unsigned)p.rows, (unsigned)p.S);
   const int pst = prefer_shared_memory();
   if (pst != ERSD_OK) return pst;
+  snprintf(g_last_launch, sizeof g_last_launch, "ersd_race_kernel<%s>%s: %d threads x (%d, %d, %d) blocks, %d chunk(s) per row",
+           dt == ERSD_BF16 ? "bf16" : "f32", many ? " (pooled thresholds)" : "", p.threads, p.B, p.rows, p.S, p.S);
   if (many) {
     if (p.threads == 128) {
       if (dt == ERSD_BF16)
@@ -521,6 +525,8 @@ static int launch_cluster_dt(const ersd_opts& o, const Params& p, cudaStream_t s
   at.val.clusterDim.z = 1;
   cfg.attrs = &at;
   cfg.numAttrs = 1;
+  snprintf(g_last_launch, sizeof g_last_launch, "ersd_cluster_kernel<%s, %d row(s) per position>: clusters of %d x %d threads, %d positions",
+           DT == ERSD_BF16 ? "bf16" : "f32", roles, CL, b256::kThreads, p.B * p.rows);
   const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, p);
   return e == cudaSuccess ? ERSD_OK : cuda_fail(e);
 }
@@ -977,6 +983,8 @@ const char* ersd_status_string(int status) {
 
 int ersd_last_cuda_error(void) { return g_last_cuda_error; }
 
-int ersd_version(void) { return 109; }
+const char* ersd_last_launch(void) { return g_last_launch; }
+
+int ersd_version(void) { return 110; }
 
 }  // extern "C"
