@@ -81,7 +81,7 @@ typedef enum {
   ERSD_ENOALLOC_LIMIT = -6 /* ersd_verify_noalloc: B * (k + 1) > ERSD_NOALLOC_MAX_ROWS */
 } ersd_status;
 
-#define ERSD_MAX_TOP_C 32   /* arrivals per race (children per tree node, opts->top_c) */
+#define ERSD_MAX_TOP_C 64   /* arrivals per race (children per tree node, opts->top_c) */
 #define ERSD_MAX_ROWS 256   /* rows per sequence: k + 1, N + 1 */
 #define ERSD_MAX_SPLIT 32   /* thread blocks sharing one row */
 #define ERSD_NOALLOC_MAX_ROWS 1024 /* ersd_verify_noalloc: largest B * (k + 1) */

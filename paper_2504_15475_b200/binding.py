@@ -18,7 +18,7 @@ LIB_PATH = os.environ.get("ERSD_LIBRARY") or os.path.join(_HERE, "libersd.so")  
 
 ERSD_F32, ERSD_BF16 = 0, 1
 ERSD_OK = 0
-ERSD_MAX_TOP_C, ERSD_MAX_ROWS, ERSD_MAX_SPLIT = 32, 256, 32
+ERSD_MAX_TOP_C, ERSD_MAX_ROWS, ERSD_MAX_SPLIT = 64, 256, 32
 ERSD_NOALLOC_MAX_ROWS = 1024
 ERSD_ENOALLOC_LIMIT = -6
 

@@ -86,7 +86,7 @@ def test_argument_errors_are_found_on_the_host(L):
     from paper_2504_15475_b200.binding import ErsdOpts
     o = ErsdOpts()
     o.struct_size = C.sizeof(ErsdOpts)
-    o.top_c = 33
+    o.top_c = 65
     assert f(p, 1, p, 1, 1, 8, 1.0, p, C.byref(o), None) == EUNSUP
     v = L.ersd_verify
     assert v(p, None, 1, p, 1, 2, 8, 1.0, p, p, None, None) == EINVAL      # k > 0 needs draft rows
@@ -102,8 +102,8 @@ def test_argument_errors_are_found_on_the_host(L):
     assert t(p, p, 1, bad_root, p, 1, 2, 8, 1.0, p, p, None, None) == EINVAL
     assert t(p, p, 1, forward, p, 1, 2, 8, 1.0, p, p, None, None) == EINVAL
     assert t(p, p, 1, good, p, 1, 2, 8, -1.0, p, p, None, None) == EINVAL
-    wide = (C.c_int32 * 35)(-1, *([0] * 34))
-    assert t(p, p, 1, wide, p, 1, 34, 8, 1.0, p, p, None, None) == EUNSUP
+    wide = (C.c_int32 * 67)(-1, *([0] * 66))                                 # 66 children: beyond ERSD_MAX_TOP_C
+    assert t(p, p, 1, wide, p, 1, 66, 8, 1.0, p, p, None, None) == EUNSUP
     o = ErsdOpts()
     o.struct_size = C.sizeof(ErsdOpts)
     o.ld_target = 4                                                          # stride below V

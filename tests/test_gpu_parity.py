@@ -423,8 +423,40 @@ def test_wide_star_uses_many_arrivals(ersd):
     assert all(len(set(r.tolist())) == 32 for r in dt)
 
 
+@pytest.mark.parametrize("c,B,V,dtype", [(64, 3, 5000, "f32"), (40, 2, 128256, "bf16"), (64, 1, 32000, "bf16")])
+def test_batch_drafting_with_up_to_64_alternatives(ersd, c, B, V, dtype):
+    """Batch drafting (Section 3: the first k arrivals under Q) with more alternatives than a warp
+    has lanes: the star's children carry the first c arrivals in order, all distinct, and the walk
+    accepts iff the target winner is among them."""
+    parent = wl.star_parent(c)
+    w = wl.Workload("star", B=B, k=c, V=V, dtype=dtype, sigma=0.5, T=1.0, config_id=53, parent=tuple(parent))
+    inp = wl.make_inputs(w)
+    out = run_verify(ersd, inp)
+    check_verify(inp, out)
+    dt = out["draft_tok"][:, 1:].cpu().numpy()
+    assert all(len(set(r.tolist())) == c for r in dt)
+    tt = out["target_tok"][:, 0].cpu().numpy()
+    acc = out["accept_len"].cpu().numpy()
+    assert ((dt == tt[:, None]).any(axis=1) == (acc == 1)).all()
+    # the near-tie counter needs one more arrival than the race wants: 63 children are the most it takes
+    near = torch.zeros(1, dtype=torch.int32, device="cuda")
+    d = to_dev(inp)
+    tok = torch.empty_like(out["tokens"])
+    al = torch.empty_like(out["accept_len"])
+    if c == 64:
+        with pytest.raises(ersd.ErsdError) as e:
+            ersd.ersd_verify_tree(d["target"], d["draft"], parent, d["seeds"], 1.0, tok, al,
+                                  ersd.make_opts(near_tie_count=near))
+        assert e.value.status == -3
+    else:
+        ersd.ersd_verify_tree(d["target"], d["draft"], parent, d["seeds"], 1.0, tok, al,
+                              ersd.make_opts(near_tie_count=near))
+        torch.cuda.synchronize()
+        assert (tok == out["tokens"]).all() and (al == out["accept_len"]).all()
+
+
 # ------------------------------------------------------------------ race sampling
-@pytest.mark.parametrize("c,split", [(1, 0), (1, 3), (4, 0), (4, 2), (32, 0), (32, 2)])
+@pytest.mark.parametrize("c,split", [(1, 0), (1, 3), (4, 0), (4, 2), (32, 0), (32, 2), (33, 0), (48, 3), (64, 0)])
 def test_race_sample_first_arrivals(ersd, c, split):
     B, R, V = 3, 4, 33000
     g = torch.Generator().manual_seed(c)
@@ -438,7 +470,7 @@ def test_race_sample_first_arrivals(ersd, c, split):
 
 
 @pytest.mark.parametrize("threads", [128, 256])
-@pytest.mark.parametrize("c,split", [(2, 1), (8, 0), (8, 7), (32, 2), (32, 16)])
+@pytest.mark.parametrize("c,split", [(2, 1), (8, 0), (8, 7), (32, 2), (32, 16), (40, 0), (64, 0), (64, 5)])
 def test_many_arrivals_at_full_vocabulary(ersd, c, split, threads):
     """Batch drafting's first c arrivals over 128256 tokens: chunks of many tiles, thresholds that
     start from the block-wide c-th smallest screening key, survivors decided several at a time."""
