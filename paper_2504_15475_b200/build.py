@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 SRC = [os.path.join(HERE, "csrc", "ersd.cu"), os.path.join(HERE, "csrc", "ersd_tree.cpp")]
-DEPS = SRC + [os.path.join(HERE, "csrc", "ersd_math.cuh"), os.path.join(HERE, "csrc", "ersd_kernel.inc"), os.path.join(HERE, "csrc", "ersd_cluster.inc"), os.path.join(HERE, "csrc", "ersd_gsd.inc"), os.path.join(ROOT, "include", "ersd.h")]
+DEPS = SRC + [os.path.join(HERE, "csrc", "ersd_math.cuh"), os.path.join(HERE, "csrc", "ersd_kernel.inc"), os.path.join(HERE, "csrc", "ersd_cluster.inc"), os.path.join(HERE, "csrc", "ersd_cluster_top.inc"), os.path.join(HERE, "csrc", "ersd_gsd.inc"), os.path.join(ROOT, "include", "ersd.h")]
 LIB = os.path.join(HERE, "libersd.so")
 
 

@@ -116,6 +116,7 @@ constexpr bool kMany = true;
 }  // namespace b128m
 namespace b256 {
 #include "ersd_cluster.inc"
+#include "ersd_cluster_top.inc"
 }  // namespace b256
 
 template <int DT>
@@ -400,13 +401,18 @@ static int launch(const Params& p, const TreeDesc& tree, int dt, bool many, cuda
 // rows of 128256 logits) or 768 (verification: two rows per position; 96 positions); beyond that
 // the streaming kernel's throughput wins (measured at V = 128256 and 32000).
 constexpr int64_t kClusterAutoBlocksSample = 1280, kClusterAutoBlocksVerify = 768;
-constexpr size_t kClusterSmemBytes = 200 * 1024;  // dynamic shared memory a block of the cluster kernel may use
+// The same for races of several arrivals (ersd_cluster_top.inc; three blocks per SM).
+constexpr int64_t kClusterAutoBlocksTop = 444;
+// dynamic shared memory a block of the cluster kernels may use (the kernel for several arrivals
+// keeps more of its lists in static shared memory)
+constexpr size_t kClusterSmemBytes = 200 * 1024, kClusterTopSmemBytes = 160 * 1024;
 
-// Tiles per block that fit (roles = rows raced together: 1, or 2 for a draft/target pair).
-static int cluster_max_tiles(int dt, int roles) {
+// Tiles per block that fit (roles = rows raced together: 1, or 2 for a draft/target pair; top:
+// the kernel for races of several arrivals).
+static int cluster_max_tiles(int dt, int roles, bool top) {
   const size_t per_tile = dt == ERSD_BF16 ? b256::cluster_role_bytes<ERSD_BF16>(1) : b256::cluster_role_bytes<ERSD_F32>(1);
-  return (int)(kClusterSmemBytes / (per_tile * (size_t)roles));
-}  // default: rows per call up to which the cluster kernel is taken
+  return (int)((top ? kClusterTopSmemBytes : kClusterSmemBytes) / (per_tile * (size_t)roles));
+}
 
 // Largest cluster (a power of two) the device takes for the cluster kernels: 16 where the opt-in
 // for non-portable sizes is granted and such a cluster fits, else 8.  Asked once per device.
@@ -419,18 +425,22 @@ static int cluster_limit(int* out) {
   if (dev < 0 || dev >= 64) return ERSD_EUNSUPPORTED;
   std::lock_guard<std::mutex> lock(m);
   if (!limit[dev]) {
-    const void* kernels[4] = {(const void*)b256::ersd_cluster_kernel<ERSD_BF16, 1>,
-                              (const void*)b256::ersd_cluster_kernel<ERSD_F32, 1>,
-                              (const void*)b256::ersd_cluster_kernel<ERSD_BF16, 2>,
-                              (const void*)b256::ersd_cluster_kernel<ERSD_F32, 2>};
-    const int smem[4] = {(int)kClusterSmemBytes, (int)kClusterSmemBytes, (int)kClusterSmemBytes,
-                         (int)kClusterSmemBytes};
+    constexpr int kKernels = 8;
+    const void* kernels[kKernels] = {(const void*)b256::ersd_cluster_kernel<ERSD_BF16, 1>,
+                                     (const void*)b256::ersd_cluster_kernel<ERSD_F32, 1>,
+                                     (const void*)b256::ersd_cluster_kernel<ERSD_BF16, 2>,
+                                     (const void*)b256::ersd_cluster_kernel<ERSD_F32, 2>,
+                                     (const void*)b256::ersd_cluster_top_kernel<ERSD_BF16, 1>,
+                                     (const void*)b256::ersd_cluster_top_kernel<ERSD_F32, 1>,
+                                     (const void*)b256::ersd_cluster_top_kernel<ERSD_BF16, 2>,
+                                     (const void*)b256::ersd_cluster_top_kernel<ERSD_F32, 2>};
     int lim = 16;
-    for (int q = 0; q < 4; ++q) {
-      e = cudaFuncSetAttribute(kernels[q], cudaFuncAttributeMaxDynamicSharedMemorySize, smem[q]);
+    for (int q = 0; q < kKernels; ++q) {
+      const int smem = (int)(q < 4 ? kClusterSmemBytes : kClusterTopSmemBytes);
+      e = cudaFuncSetAttribute(kernels[q], cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
       if (e != cudaSuccess) return cuda_fail(e);
     }
-    for (int q = 0; q < 4 && lim == 16; ++q) {
+    for (int q = 0; q < kKernels && lim == 16; ++q) {
       e = cudaFuncSetAttribute(kernels[q], cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
       int n = 0;
       if (e == cudaSuccess) {
@@ -438,7 +448,7 @@ static int cluster_limit(int* out) {
         memset(&cfg, 0, sizeof cfg);
         cfg.gridDim = dim3(16, 1, 1);
         cfg.blockDim = dim3(b256::kThreads, 1, 1);
-        cfg.dynamicSmemBytes = (size_t)smem[q];
+        cfg.dynamicSmemBytes = q < 4 ? kClusterSmemBytes : kClusterTopSmemBytes;
         cudaLaunchAttribute at;
         at.id = cudaLaunchAttributeClusterDimension;
         at.val.clusterDim.x = 16;
@@ -457,27 +467,32 @@ static int cluster_limit(int* out) {
   return ERSD_OK;
 }
 
-// Whether a sampling call can take the cluster kernel at all.
-static bool cluster_applies(const Params& p, int dt) {
+// Whether a call can take a cluster kernel at all; cmax: most arrivals any of its races wants.
+static bool cluster_applies(const Params& p, int dt, int cmax) {
   // (eight blocks, the portable cluster size, must be able to stage the rows of a position)
+  const bool top = cmax > 1;
   const int roles = (p.mode == kVerify && p.draft) ? 2 : 1;
   const int64_t ntiles = ((int64_t)p.V + b256::kTile - 1) / b256::kTile;
-  if (ntiles > 8 * (int64_t)cluster_max_tiles(dt, roles)) return false;
-  if (p.mode == kVerify && p.rows > 32) return false;
-  return p.c_sample == 1 && p.aligned_t && (roles == 1 || p.aligned_d) && p.rows <= 65535 && p.B <= 65535;
+  if (ntiles > 8 * (int64_t)cluster_max_tiles(dt, roles, top)) return false;
+  if (top) {
+    if (cmax > b256::kTopMaxC || p.given_tok || p.chain_outputs || p.extra) return false;
+  } else if (p.mode == kVerify && p.rows > 32) {
+    return false;
+  }
+  return p.aligned_t && (roles == 1 || p.aligned_d) && p.rows <= 65535 && p.B <= 65535;
 }
 
 // Blocks per cluster.  Few positions: the smallest power of two that leaves a block about
 // kClusterGroups tiles (shortest path through one position).  Once such clusters would make more
 // than two blocks per SM: blocks of about twice as many tiles (measured at V = 128256: clusters
 // of 8 beat clusters of 16 from about 20 positions on, clusters of 4 never beat clusters of 8).
-static int cluster_size(const ersd_opts& o, const Params& p, int dt, int* out) {
+static int cluster_size(const ersd_opts& o, const Params& p, int dt, int cmax, int* out) {
   int lim = 8;
   const int ls = cluster_limit(&lim);
   if (ls != ERSD_OK) return ls;
   const int ntiles = (p.V + b256::kTile - 1) / b256::kTile;
   const int roles = (p.mode == kVerify && p.draft) ? 2 : 1;
-  const int max_tiles = cluster_max_tiles(dt, roles);
+  const int max_tiles = cluster_max_tiles(dt, roles, cmax > 1);
   if (o.split_v) {  // the caller's choice: a power of two that the device takes and whose blocks can stage their share
     const int CL = (int)o.split_v;
     if (CL > lim || (CL & (CL - 1)) != 0 || (ntiles + CL - 1) / CL > max_tiles) return ERSD_EUNSUPPORTED;
@@ -495,20 +510,20 @@ static int cluster_size(const ersd_opts& o, const Params& p, int dt, int* out) {
 }
 
 // Whether a call that leaves the choice to the library takes the cluster kernel.
-static bool cluster_by_default(const ersd_opts& o, const Params& p, int dt) {
-  if (o.kernel_path != 0 || o.split_v != 0 || o.block_threads != 0 || !cluster_applies(p, dt)) return false;
+static bool cluster_by_default(const ersd_opts& o, const Params& p, int dt, int cmax) {
+  if (o.kernel_path != 0 || o.split_v != 0 || o.block_threads != 0 || !cluster_applies(p, dt, cmax)) return false;
   int CL = 1;
-  if (cluster_size(o, p, dt, &CL) != ERSD_OK) return false;
+  if (cluster_size(o, p, dt, cmax, &CL) != ERSD_OK) return false;
   const int64_t blocks = (int64_t)p.B * p.rows * CL;
+  if (cmax > 1) return blocks <= kClusterAutoBlocksTop;
   return blocks <= (p.mode == kVerify ? kClusterAutoBlocksVerify : kClusterAutoBlocksSample);
 }
 
 template <int DT>
-static int launch_cluster_dt(const ersd_opts& o, const Params& p, cudaStream_t st) {
+static int launch_cluster_dt(const ersd_opts& o, const Params& p, const TreeDesc& tree, int cmax, cudaStream_t st) {
   const int roles = (p.mode == kVerify && p.draft) ? 2 : 1;
-  auto kernel = roles == 2 ? b256::ersd_cluster_kernel<DT, 2> : b256::ersd_cluster_kernel<DT, 1>;
   int CL = 1;
-  const int ls = cluster_size(o, p, DT, &CL);
+  const int ls = cluster_size(o, p, DT, cmax, &CL);
   if (ls != ERSD_OK) return ls;
   const int ntiles = (p.V + b256::kTile - 1) / b256::kTile;
   const int G = (ntiles + CL - 1) / CL;  // tiles per block; they fit, see cluster_applies
@@ -525,14 +540,23 @@ static int launch_cluster_dt(const ersd_opts& o, const Params& p, cudaStream_t s
   at.val.clusterDim.z = 1;
   cfg.attrs = &at;
   cfg.numAttrs = 1;
-  snprintf(g_last_launch, sizeof g_last_launch, "ersd_cluster_kernel<%s, %d row(s) per position>: clusters of %d x %d threads, %d positions",
-           DT == ERSD_BF16 ? "bf16" : "f32", roles, CL, b256::kThreads, p.B * p.rows);
-  const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, p);
+  snprintf(g_last_launch, sizeof g_last_launch, "%s<%s, %d row(s) per position>: clusters of %d x %d threads, %d positions",
+           cmax > 1 ? "ersd_cluster_top_kernel" : "ersd_cluster_kernel", DT == ERSD_BF16 ? "bf16" : "f32", roles, CL,
+           b256::kThreads, p.B * p.rows);
+  cudaError_t e;
+  if (cmax > 1) {
+    auto kernel = roles == 2 ? b256::ersd_cluster_top_kernel<DT, 2> : b256::ersd_cluster_top_kernel<DT, 1>;
+    e = cudaLaunchKernelEx(&cfg, kernel, p, tree);
+  } else {
+    auto kernel = roles == 2 ? b256::ersd_cluster_kernel<DT, 2> : b256::ersd_cluster_kernel<DT, 1>;
+    e = cudaLaunchKernelEx(&cfg, kernel, p);
+  }
   return e == cudaSuccess ? ERSD_OK : cuda_fail(e);
 }
 
-static int launch_cluster(const ersd_opts& o, const Params& p, int dt, cudaStream_t st) {
-  return dt == ERSD_BF16 ? launch_cluster_dt<ERSD_BF16>(o, p, st) : launch_cluster_dt<ERSD_F32>(o, p, st);
+static int launch_cluster(const ersd_opts& o, const Params& p, const TreeDesc& tree, int dt, int cmax, cudaStream_t st) {
+  return dt == ERSD_BF16 ? launch_cluster_dt<ERSD_BF16>(o, p, tree, cmax, st)
+                         : launch_cluster_dt<ERSD_F32>(o, p, tree, cmax, st);
 }
 
 static int check_common(const void* logits, int dt, const uint64_t* seeds, int B, int rows, int V,
@@ -596,10 +620,10 @@ static int verify_impl(const void* target, const void* draft, int dt, const Tree
   if (((uintptr_t)o.near_tie_count & 3) != 0) return ERSD_EALIGN;
   if (cmax + p.extra > ERSD_MAX_TOP_C) return ERSD_EUNSUPPORTED;
   cmax += p.extra;
-  // sequences of few rows: one cluster per position (chains only: one arrival per race; near-ties
-  // are counted by the streaming kernel only, the cluster kernel keeps no runner-up key)
+  // sequences of few rows: one cluster per position (near-ties are counted by the streaming
+  // kernel only: the cluster kernels keep no arrival beyond those asked for)
   if (o.kernel_path > 2) return ERSD_EINVAL;
-  const bool cluster_ok = cmax <= 1 && cluster_applies(p, dt);  // (a tree without branching is the chain 0 -> 1 -> ...)
+  const bool cluster_ok = !p.extra && cluster_applies(p, dt, cmax);  // (a tree without branching is the chain 0 -> 1 -> ...)
   if (o.kernel_path == 2 && !cluster_ok) return ERSD_EUNSUPPORTED;
   if (o.block_threads != 0 && o.block_threads != 128 && o.block_threads != 256) return ERSD_EINVAL;
   if (o.workspace) {
@@ -611,8 +635,8 @@ static int verify_impl(const void* target, const void* draft, int dt, const Tree
   const int st = get_workspace(o, workspace_bytes(B, rows), &ws, (cudaStream_t)stream);
   if (st != ERSD_OK) return st;
   p.slots = (Slot*)ws;
-  if (cluster_ok && (o.kernel_path == 2 || cluster_by_default(o, p, dt)))
-    return launch_cluster(o, p, dt, (cudaStream_t)stream);
+  if (cluster_ok && (o.kernel_path == 2 || cluster_by_default(o, p, dt, cmax)))
+    return launch_cluster(o, p, tree, dt, cmax, (cudaStream_t)stream);
   int st0 = choose_threads(o, (int64_t)B * rows, &p.threads);
   if (st0 != ERSD_OK) return st0;
   set_chunks(p, choose_split(o, (int64_t)B * rows, V, cmax, p.threads));
@@ -732,10 +756,13 @@ int ersd_race_sample(const void* logits, ersd_dtype dt, const uint64_t* seeds, i
   p.near_tie = o.near_tie_count;
   p.extra = extra;
   if (o.kernel_path > 2) return ERSD_EINVAL;
-  // (near-ties are counted by the streaming kernel only: the cluster kernel keeps no runner-up key)
-  const bool cluster_ok = !extra && cluster_applies(p, dt);
+  // (near-ties are counted by the streaming kernel only: the cluster kernels keep no arrival beyond those asked for)
+  const bool cluster_ok = !extra && cluster_applies(p, dt, c);
   if (o.kernel_path == 2 && !cluster_ok) return ERSD_EUNSUPPORTED;
-  if (cluster_ok && (o.kernel_path == 2 || cluster_by_default(o, p, dt))) return launch_cluster(o, p, dt, (cudaStream_t)cuda_stream);
+  TreeDesc tree;
+  memset(&tree, 0, sizeof tree);
+  if (cluster_ok && (o.kernel_path == 2 || cluster_by_default(o, p, dt, c)))
+    return launch_cluster(o, p, tree, dt, c, (cudaStream_t)cuda_stream);
   st = choose_threads(o, (int64_t)B * R, &p.threads);
   if (st != ERSD_OK) return st;
   set_chunks(p, choose_split(o, (int64_t)B * R, V, c + extra, p.threads));
@@ -745,8 +772,6 @@ int ersd_race_sample(const void* logits, ersd_dtype dt, const uint64_t* seeds, i
     if (st != ERSD_OK) return st;
     p.slots = (Slot*)ws;
   }
-  TreeDesc tree;
-  memset(&tree, 0, sizeof tree);
   return launch(p, tree, dt, c + extra > 1, (cudaStream_t)cuda_stream);
 }
 

@@ -65,14 +65,46 @@ def time_trees(args):
             acc = torch.empty(B, dtype=torch.int32, device="cuda")
             ws = torch.zeros(binding.ersd_workspace_bytes(B, n), dtype=torch.uint8, device="cuda")
             binding.ersd_workspace_init(ws)
-            opts = binding.make_opts(workspace=ws, split_v=args.split)
+            for kernel, path in PATHS.items():
+                opts = binding.make_opts(workspace=ws, kernel_path=path, split_v=args.split if path else 0)
 
-            def call(i, st):
-                t, d = sets[i % len(sets)]
-                binding.ersd_verify_tree(t, d, parent, seeds, 1.0, tok, acc, opts, st)
+                def call(i, st):
+                    t, d = sets[i % len(sets)]
+                    binding.ersd_verify_tree(t, d, parent, seeds, 1.0, tok, acc, opts, st)
 
-            print(json.dumps({"entry": "ersd_verify_tree", "tree": name, "nodes": n, "B": B, "V": V, "dtype": "bf16",
-                              "us_per_call": round(graph_time_us(call), 2),
+                try:
+                    call(0, torch.cuda.current_stream())
+                except binding.ErsdError:                     # this kernel does not take the call
+                    continue
+                print(json.dumps({"entry": "ersd_verify_tree", "tree": name, "nodes": n, "B": B, "V": V,
+                                  "dtype": "bf16", "kernel": kernel, "launch": binding.ersd_last_launch(),
+                                  "us_per_call": round(graph_time_us(call), 2),
+                                  "timing": "CUDA graph replay, 30 calls per graph"}), flush=True)
+
+
+def time_batch_drafting(args, c=8):
+    """ersd_race_sample with top_c = c: the first c arrivals of one race per sequence."""
+    V = args.V
+    for B in [int(x) for x in args.batches.split(",")]:
+        gen = torch.Generator().manual_seed(3000 + B)
+        rows = [wl.zipf_rows(B, V, gen, "cpu").view(B, 1, V).to(torch.bfloat16).cuda() for _ in range(min(args.sets, 4))]
+        seeds = wl.make_seeds(79, B, B).cuda()
+        tok = torch.empty(B, 1, c, dtype=torch.int32, device="cuda")
+        ws = torch.zeros(binding.ersd_workspace_bytes(B, 1), dtype=torch.uint8, device="cuda")
+        binding.ersd_workspace_init(ws)
+        for kernel, path in PATHS.items():
+            opts = binding.make_opts(workspace=ws, kernel_path=path, top_c=c, split_v=args.split if path else 0)
+
+            def draft(i, st):
+                binding.ersd_race_sample(rows[i % len(rows)], seeds, 1.0, tok, opts, st)
+
+            try:
+                draft(0, torch.cuda.current_stream())
+            except binding.ErsdError:                         # this kernel does not take the call
+                continue
+            print(json.dumps({"entry": "ersd_race_sample", "top_c": c, "B": B, "V": V, "dtype": "bf16",
+                              "kernel": kernel, "launch": binding.ersd_last_launch(),
+                              "us_per_call": round(graph_time_us(draft), 2),
                               "timing": "CUDA graph replay, 30 calls per graph"}), flush=True)
 
 
@@ -84,7 +116,7 @@ def main():
     ap.add_argument("--sets", type=int, default=6, help="distinct inputs rotated between calls")
     ap.add_argument("--split", type=int, default=0, help="thread blocks per row / per cluster (0: library default)")
     ap.add_argument("--trees", action="store_true",
-                    help="time ersd_verify_tree on draft trees (streaming kernel) instead of the two entries above")
+                    help="time ersd_verify_tree on draft trees, and batch drafting, instead of the two entries above")
     ap.add_argument("--plain", type=int, default=0,
                     help="issue this many plain calls per case instead of replaying a graph and print no "
                          "times (for a profiler's launch list)")
@@ -95,6 +127,7 @@ def main():
     V, k = args.V, args.k
     if args.trees:
         time_trees(args)
+        time_batch_drafting(args)
         return
     for B in [int(x) for x in args.batches.split(",")]:
         gen = torch.Generator().manual_seed(1000 + B)

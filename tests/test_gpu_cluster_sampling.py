@@ -147,13 +147,13 @@ def test_where_the_cluster_kernel_does_not_apply(ersd):
     B, R, V = 2, 2, 1003
     logits = torch.randn(B, R, V).to(torch.bfloat16).cuda()      # rows of 2006 bytes: not 16-byte aligned
     seeds = wl.make_seeds(1, 0, B).cuda()
-    tok = torch.empty(B, R, 4, dtype=torch.int32, device="cuda")
+    tok = torch.empty(B, R, 33, dtype=torch.int32, device="cuda")
     with pytest.raises(ersd.ErsdError) as e:
         ersd.ersd_race_sample(logits, seeds, 1.0, tok, ersd.make_opts(kernel_path=CLUSTER))
     assert e.value.status == -3
     ok = torch.randn(B, R, 1024).to(torch.bfloat16).cuda()
-    with pytest.raises(ersd.ErsdError) as e:
-        ersd.ersd_race_sample(ok, seeds, 1.0, tok, ersd.make_opts(kernel_path=CLUSTER, top_c=4))
+    with pytest.raises(ersd.ErsdError) as e:   # (up to 32 arrivals per race take the cluster kernel of their own)
+        ersd.ersd_race_sample(ok, seeds, 1.0, tok, ersd.make_opts(kernel_path=CLUSTER, top_c=33))
     assert e.value.status == -3
     with pytest.raises(ersd.ErsdError) as e:
         ersd.ersd_race_sample(ok, seeds, 1.0, tok, ersd.make_opts(kernel_path=3))

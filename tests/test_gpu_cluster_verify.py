@@ -242,8 +242,8 @@ def test_a_chain_given_as_a_tree(ersd):
 def test_where_the_cluster_kernel_does_not_apply(ersd):
     B, V = 2, 1024
     seeds = wl.make_seeds(1, 0, B).cuda()
-    # trees: several arrivals per race
-    parent = wl.star_parent(3)
+    # trees whose races want more than 32 arrivals
+    parent = wl.star_parent(33)
     t = torch.randn(B, len(parent), V).to(torch.bfloat16).cuda()
     tok = torch.empty(B, 2, dtype=torch.int32, device="cuda")
     acc = torch.empty(B, dtype=torch.int32, device="cuda")
