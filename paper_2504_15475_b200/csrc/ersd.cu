@@ -85,6 +85,7 @@ struct Params {
   float* out_key;        // sample mode
   uint32_t* near_tie;    // count of races with two consecutive arrivals closer than 1e-5 (nullable)
   int extra;             // 1 when near-ties are counted: every race is run for one more arrival
+  int top_cmax;          // cluster kernel for several arrivals: most arrivals any race of the call wants
   Slot* slots;
 };
 
@@ -403,15 +404,14 @@ static int launch(const Params& p, const TreeDesc& tree, int dt, bool many, cuda
 constexpr int64_t kClusterAutoBlocksSample = 1280, kClusterAutoBlocksVerify = 768;
 // The same for races of several arrivals (ersd_cluster_top.inc; three blocks per SM).
 constexpr int64_t kClusterAutoBlocksTop = 444;
-// dynamic shared memory a block of the cluster kernels may use (the kernel for several arrivals
-// keeps more of its lists in static shared memory)
-constexpr size_t kClusterSmemBytes = 200 * 1024, kClusterTopSmemBytes = 160 * 1024;
+constexpr size_t kClusterSmemBytes = 200 * 1024;  // dynamic shared memory a block of the cluster kernels may use
 
-// Tiles per block that fit (roles = rows raced together: 1, or 2 for a draft/target pair; top:
-// the kernel for races of several arrivals).
-static int cluster_max_tiles(int dt, int roles, bool top) {
+// Tiles per block that fit (roles = rows raced together: 1, or 2 for a draft/target pair; cmax > 1:
+// the kernel for races of several arrivals, which keeps its lists behind the rows).
+static int cluster_max_tiles(int dt, int roles, int cmax) {
   const size_t per_tile = dt == ERSD_BF16 ? b256::cluster_role_bytes<ERSD_BF16>(1) : b256::cluster_role_bytes<ERSD_F32>(1);
-  return (int)((top ? kClusterTopSmemBytes : kClusterSmemBytes) / (per_tile * (size_t)roles));
+  const size_t lists = cmax > 1 ? b256::top_list_bytes(cmax, b256::kClusterMax) : 0;
+  return (int)((kClusterSmemBytes - lists) / (per_tile * (size_t)roles));
 }
 
 // Largest cluster (a power of two) the device takes for the cluster kernels: 16 where the opt-in
@@ -436,8 +436,7 @@ static int cluster_limit(int* out) {
                                      (const void*)b256::ersd_cluster_top_kernel<ERSD_F32, 2>};
     int lim = 16;
     for (int q = 0; q < kKernels; ++q) {
-      const int smem = (int)(q < 4 ? kClusterSmemBytes : kClusterTopSmemBytes);
-      e = cudaFuncSetAttribute(kernels[q], cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+      e = cudaFuncSetAttribute(kernels[q], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kClusterSmemBytes);
       if (e != cudaSuccess) return cuda_fail(e);
     }
     for (int q = 0; q < kKernels && lim == 16; ++q) {
@@ -448,7 +447,7 @@ static int cluster_limit(int* out) {
         memset(&cfg, 0, sizeof cfg);
         cfg.gridDim = dim3(16, 1, 1);
         cfg.blockDim = dim3(b256::kThreads, 1, 1);
-        cfg.dynamicSmemBytes = q < 4 ? kClusterSmemBytes : kClusterTopSmemBytes;
+        cfg.dynamicSmemBytes = kClusterSmemBytes;
         cudaLaunchAttribute at;
         at.id = cudaLaunchAttributeClusterDimension;
         at.val.clusterDim.x = 16;
@@ -473,9 +472,10 @@ static bool cluster_applies(const Params& p, int dt, int cmax) {
   const bool top = cmax > 1;
   const int roles = (p.mode == kVerify && p.draft) ? 2 : 1;
   const int64_t ntiles = ((int64_t)p.V + b256::kTile - 1) / b256::kTile;
-  if (ntiles > 8 * (int64_t)cluster_max_tiles(dt, roles, top)) return false;
+  if (top && cmax > b256::kTopMaxC) return false;
+  if (ntiles > 8 * (int64_t)cluster_max_tiles(dt, roles, cmax)) return false;
   if (top) {
-    if (cmax > b256::kTopMaxC || p.given_tok || p.chain_outputs || p.extra) return false;
+    if (p.given_tok || p.chain_outputs || p.extra) return false;
   } else if (p.mode == kVerify && p.rows > 32) {
     return false;
   }
@@ -492,7 +492,7 @@ static int cluster_size(const ersd_opts& o, const Params& p, int dt, int cmax, i
   if (ls != ERSD_OK) return ls;
   const int ntiles = (p.V + b256::kTile - 1) / b256::kTile;
   const int roles = (p.mode == kVerify && p.draft) ? 2 : 1;
-  const int max_tiles = cluster_max_tiles(dt, roles, cmax > 1);
+  const int max_tiles = cluster_max_tiles(dt, roles, cmax);
   if (o.split_v) {  // the caller's choice: a power of two that the device takes and whose blocks can stage their share
     const int CL = (int)o.split_v;
     if (CL > lim || (CL & (CL - 1)) != 0 || (ntiles + CL - 1) / CL > max_tiles) return ERSD_EUNSUPPORTED;
@@ -520,7 +520,9 @@ static bool cluster_by_default(const ersd_opts& o, const Params& p, int dt, int 
 }
 
 template <int DT>
-static int launch_cluster_dt(const ersd_opts& o, const Params& p, const TreeDesc& tree, int cmax, cudaStream_t st) {
+static int launch_cluster_dt(const ersd_opts& o, const Params& p_in, const TreeDesc& tree, int cmax, cudaStream_t st) {
+  Params p = p_in;
+  p.top_cmax = cmax;
   const int roles = (p.mode == kVerify && p.draft) ? 2 : 1;
   int CL = 1;
   const int ls = cluster_size(o, p, DT, cmax, &CL);
@@ -531,7 +533,7 @@ static int launch_cluster_dt(const ersd_opts& o, const Params& p, const TreeDesc
   memset(&cfg, 0, sizeof cfg);
   cfg.gridDim = dim3((unsigned)CL, (unsigned)p.rows, (unsigned)p.B);
   cfg.blockDim = dim3(b256::kThreads, 1, 1);
-  cfg.dynamicSmemBytes = b256::cluster_role_bytes<DT>(G) * (size_t)roles;
+  cfg.dynamicSmemBytes = b256::cluster_role_bytes<DT>(G) * (size_t)roles + (cmax > 1 ? b256::top_list_bytes(cmax, CL) : 0);
   cfg.stream = st;
   cudaLaunchAttribute at;
   at.id = cudaLaunchAttributeClusterDimension;
