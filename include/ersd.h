@@ -109,21 +109,24 @@ typedef struct ersd_opts {
   float* out_key;          /* device, nullable, ersd_race_sample: [B, R, c] keys of the arrivals */
   void* workspace;         /* device scratch or NULL (library-owned) */
   size_t workspace_bytes;
-  uint32_t kernel_path;    /* ersd_race_sample, ersd_verify, ersd_verify_tokens, ersd_verify_noalloc, and
-                              ersd_verify_tree on a tree without branching:
-                              0 = chosen by the library, 1 = the streaming kernel, 2 = the cluster kernel
-                              (one thread-block cluster per position, for calls of few rows;
-                              ERSD_EUNSUPPORTED where it does not apply: top_c > 1, a node with several
-                              children, rows not 16-byte aligned, B or R > 65535, more than 32 rows per
-                              sequence, or a vocabulary too long for eight
-                              blocks to stage in shared memory: beyond about 320 k entries in bf16,
-                              160 k in fp32, halved when draft rows are raced along) */
+  uint32_t kernel_path;    /* ersd_race_sample, ersd_verify, ersd_verify_tokens, ersd_verify_noalloc,
+                              ersd_verify_tree:
+                              0 = chosen by the library, 1 = the streaming kernel, 2 = a cluster kernel
+                              (one thread-block cluster per position, for calls of few rows; one kernel for
+                              races of one arrival, one for races of up to 32: top_c > 1, trees with
+                              branching;
+                              ERSD_EUNSUPPORTED where neither applies: a race of more than 32 arrivals,
+                              rows not 16-byte aligned, B or R > 65535, more than 32 rows per sequence
+                              in ersd_verify and its variants, near_tie_count given, or a vocabulary too
+                              long for eight blocks to stage in shared memory: beyond about 320 k entries
+                              in bf16, 160 k in fp32, halved when draft rows are raced along, less the
+                              room the lists of a race of several arrivals take) */
   uint32_t reserved1;
   uint32_t* near_tie_count; /* device, nullable: a counter the call ADDS to (the caller zeroes it): the number
                               of races in which two consecutive arrivals among the first c + 1 (c = arrivals
                               wanted: 1 for a winner, a node's child count for its draft row, top_c) have race
-                              keys closer than 1e-5 -- the benchmark spec's near-tie window, inside which a reference
-                              in other arithmetic may order the two the other way.  To see the runner-up every
+                              keys closer than 1e-5 -- the window inside which a reference in other arithmetic
+                              may order the two the other way.  To see the runner-up every
                               race is run for one more arrival (c + 1 <= ERSD_MAX_TOP_C, else
                               ERSD_EUNSUPPORTED), which costs time, and the call takes the streaming kernel
                               (kernel_path 2 is refused).  Leave NULL in production. */

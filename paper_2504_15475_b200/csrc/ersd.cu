@@ -403,7 +403,7 @@ static int launch(const Params& p, const TreeDesc& tree, int dt, bool many, cuda
 // the streaming kernel's throughput wins (measured at V = 128256 and 32000).
 constexpr int64_t kClusterAutoBlocksSample = 1280, kClusterAutoBlocksVerify = 768;
 // The same for races of several arrivals (ersd_cluster_top.inc; three blocks per SM).
-constexpr int64_t kClusterAutoBlocksTop = 444;
+constexpr int64_t kClusterAutoBlocksTop = 600;
 constexpr size_t kClusterSmemBytes = 200 * 1024;  // dynamic shared memory a block of the cluster kernels may use
 
 // Tiles per block that fit (roles = rows raced together: 1, or 2 for a draft/target pair; cmax > 1:
@@ -1012,6 +1012,6 @@ int ersd_last_cuda_error(void) { return g_last_cuda_error; }
 
 const char* ersd_last_launch(void) { return g_last_launch; }
 
-int ersd_version(void) { return 110; }
+int ersd_version(void) { return 111; }
 
 }  // extern "C"

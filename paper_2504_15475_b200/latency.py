@@ -1,6 +1,7 @@
 """Device time per call of small-batch race sampling and sequence verification.
 
     python -m paper_2504_15475_b200.latency [--V 128256] [--k 5] [--batches 1,2,4,8,16,32]
+    python -m paper_2504_15475_b200.latency --trees [--batches 1,2,4]     # draft trees, batch drafting
 
 Calls of a few rows are bound by latency, not by bandwidth, and a Python caller cannot issue
 them faster than about ten microseconds apart; so the calls are captured into a CUDA graph (30
@@ -76,6 +77,11 @@ def time_trees(args):
                     call(0, torch.cuda.current_stream())
                 except binding.ErsdError:                     # this kernel does not take the call
                     continue
+                if args.plain:
+                    for i in range(args.plain):
+                        call(i, torch.cuda.current_stream())
+                    torch.cuda.synchronize()
+                    continue
                 print(json.dumps({"entry": "ersd_verify_tree", "tree": name, "nodes": n, "B": B, "V": V,
                                   "dtype": "bf16", "kernel": kernel, "launch": binding.ersd_last_launch(),
                                   "us_per_call": round(graph_time_us(call), 2),
@@ -101,6 +107,11 @@ def time_batch_drafting(args, c=8):
             try:
                 draft(0, torch.cuda.current_stream())
             except binding.ErsdError:                         # this kernel does not take the call
+                continue
+            if args.plain:
+                for i in range(args.plain):
+                    draft(i, torch.cuda.current_stream())
+                torch.cuda.synchronize()
                 continue
             print(json.dumps({"entry": "ersd_race_sample", "top_c": c, "B": B, "V": V, "dtype": "bf16",
                               "kernel": kernel, "launch": binding.ersd_last_launch(),

@@ -116,8 +116,9 @@ def test_argument_errors_are_found_on_the_host(L):
     o.kernel_path = 2                                                        # the cluster kernel where it cannot run
     assert v(p, p, 1, p, 1, 32, 8, 1.0, p, p, C.byref(o), None) == EUNSUP    # more than 32 positions
     assert v(p, C.c_void_p(0x1002), 1, p, 1, 2, 8, 1.0, p, p, C.byref(o), None) == EUNSUP  # draft rows not 16-byte aligned
-    assert t(p, p, 1, good, p, 1, 2, 8, 1.0, p, p, C.byref(o), None) == EUNSUP  # two arrivals per race
-    o.top_c = 2
+    star33 = (C.c_int32 * 34)(-1, *([0] * 33))
+    assert t(p, p, 1, star33, p, 1, 33, 8, 1.0, p, p, C.byref(o), None) == EUNSUP  # more than 32 arrivals per race
+    o.top_c = 33
     assert f(p, 1, p, 1, 1, 8, 1.0, p, C.byref(o), None) == EUNSUP
     assert L.ersd_verify_tokens(p, None, 1, p, 1, 2, 8, 1.0, p, p, None, None) == EINVAL      # k > 0 needs tokens
     assert L.ersd_verify_tokens(p, C.c_void_p(4098), 1, p, 1, 2, 8, 1.0, p, p, None, None) == -2  # misaligned int32

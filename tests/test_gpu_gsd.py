@@ -4,7 +4,7 @@ oracle's Algorithms 1 and 4, through the C boundary, on the same seeded inputs.
 Bar: emitted tokens and accept lengths equal the oracle's.  Both sides decide in double precision,
 so the allowed exceptions are decisions within rounding of each other, which the oracle's outputs
 expose: a ratio test with |ratio - u| < 1e-9 * ratio, or a final race whose two best arrival times
-are closer than 1e-5 relative (the benchmark spec's near-tie window); such sequences are counted."""
+are closer than 1e-5 relative (the near-tie window); such sequences are counted."""
 import numpy as np
 import pytest
 import torch
