@@ -90,7 +90,7 @@ struct Params {
 };
 
 // ---------------------------------------------------------------------------------------------
-// The kernel, compiled for two block sizes: many rows are raced by 128-thread blocks (eight per
+// The kernel, compiled for two block sizes: many rows are raced by 128-thread blocks (seven per
 // SM: more, smaller work items and a shorter last wave), few rows by 256-thread blocks (four per
 // SM: a row's thresholds are shared by more warps, half as many blocks to set up).
 // ---------------------------------------------------------------------------------------------

@@ -192,6 +192,24 @@ def test_tree_verification(ersd, shape, B, V, dtype):
         assert same(out, verify_tree(ersd, inp, STREAMING))
 
 
+@pytest.mark.parametrize("V", [4096, 128256])
+def test_greedy_tree_over_tied_logits(ersd, V):
+    """T = 0 with draft and target rows of equal logits everywhere: both roles of a position list
+    every group (more than a block's candidate list holds), arrivals are the lowest indices, the
+    target's winner is the first child's token at every level."""
+    parent = tuple(TREES["c4"])
+    B, n = 2, len(parent)
+    t = torch.zeros(B, n, V, dtype=torch.bfloat16)
+    t[1, :, 1000:] = -3.0                                  # second sequence: ties among the first thousand only
+    inp = dict(target=t, draft=t.clone(), seeds=wl.make_seeds(83, 0, B), T=0.0, temps=None, parent=list(parent))
+    out = verify_tree(ersd, inp, CLUSTER)
+    assert "ersd_cluster_top_kernel" in ersd.ersd_last_launch()
+    check_verify(inp, out)
+    assert (out["accept_len"] == 4).all() and (out["tokens"] == 0).all()
+    assert out["draft_tok"][0, 1:5].tolist() == [0, 1, 2, 3]
+    assert same(out, verify_tree(ersd, inp, STREAMING))
+
+
 def test_tree_verification_repeats_bit_for_bit_and_leaves_the_workspace_clean(ersd):
     parent = tuple(TREES["c4"])
     w = wl.Workload("tree_rep", B=2, k=len(parent) - 1, V=128256, dtype="bf16", sigma=0.5, T=1.0, config_id=81,
