@@ -358,8 +358,11 @@ static int prefer_shared_memory() {
 // top_c > 1).  Calls of up to two rows per SM then take the variant of the kernel that pools the
 // block's decided indices (measured: a star of 8 at B=1 48 -> 42 us, the 17-node tree 35 -> 33 us;
 // at 544 rows the pooling costs 0.7 % instead).
-static int launch(const Params& p, const TreeDesc& tree, int dt, bool many, cudaStream_t st) {
-  many = many && (int64_t)p.B * p.rows <= 2 * sm_count();
+// cmax: most arrivals any race of the call wants.  The builds for races of several arrivals take
+// calls of few rows (their loop is slower, their rare path quicker) and every call with a race of
+// more than 32 arrivals (only they hold two list entries per lane).
+static int launch(const Params& p, const TreeDesc& tree, int dt, int cmax, cudaStream_t st) {
+  const bool many = cmax > 32 || (cmax > 1 && (int64_t)p.B * p.rows <= 2 * sm_count());
   // grid (sequence, row in launch order, chunk): blocks are dispatched x fastest, z slowest, which
   // is the chunk-major order the kernel counts on, and the kernel needs no division to decode
   if (p.rows > 65535 || p.S > 65535) return ERSD_EUNSUPPORTED;
@@ -642,7 +645,7 @@ static int verify_impl(const void* target, const void* draft, int dt, const Tree
   int st0 = choose_threads(o, (int64_t)B * rows, &p.threads);
   if (st0 != ERSD_OK) return st0;
   set_chunks(p, choose_split(o, (int64_t)B * rows, V, cmax, p.threads));
-  return launch(p, tree, dt, cmax > 1, (cudaStream_t)stream);
+  return launch(p, tree, dt, cmax, (cudaStream_t)stream);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -774,7 +777,7 @@ int ersd_race_sample(const void* logits, ersd_dtype dt, const uint64_t* seeds, i
     if (st != ERSD_OK) return st;
     p.slots = (Slot*)ws;
   }
-  return launch(p, tree, dt, c + extra > 1, (cudaStream_t)cuda_stream);
+  return launch(p, tree, dt, c + extra, (cudaStream_t)cuda_stream);
 }
 
 static int verify_sequence(const void* target_logits, const void* draft_logits, int dt,

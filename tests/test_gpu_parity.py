@@ -488,6 +488,29 @@ def test_many_arrivals_at_full_vocabulary(ersd, c, split, threads):
     assert all(len(set(r.tolist())) == c for r in tok.view(-1, c).cpu())
 
 
+def test_more_than_32_arrivals_in_calls_of_many_rows(ersd):
+    """Races of more than 32 arrivals need two list entries per lane, which only the builds for
+    several arrivals hold: calls of many rows (which otherwise take the other builds) must get them."""
+    B, R, V, c = 90, 4, 6000, 40                       # 360 rows
+    g = torch.Generator().manual_seed(40)
+    logits = wl.zipf_rows(B * R, V, g, "cpu").view(B, R, V).to(torch.bfloat16)
+    seeds = wl.make_seeds(18, c, B)
+    tok = torch.empty(B, R, c, dtype=torch.int32, device="cuda")
+    key = torch.empty(B, R, c, dtype=torch.float32, device="cuda")
+    ersd.ersd_race_sample(logits.cuda(), seeds.cuda(), 0.9, tok, ersd.make_opts(top_c=c, out_key=key))
+    torch.cuda.synchronize()
+    assert "pooled thresholds" in ersd.ersd_last_launch()
+    assert check_sample(logits, seeds, 0.9, tok, key, c=c) == 0
+    parent = wl.star_parent(40)                        # 41 rows per sequence, 410 in all
+    w = wl.Workload("star40_many", B=10, k=40, V=5000, dtype="bf16", sigma=0.8, T=1.0, config_id=47, parent=tuple(parent))
+    inp = wl.make_inputs(w)
+    out = ersd.verify(inp["target"].cuda(), inp["draft"].cuda(), inp["seeds"].cuda(), inp["T"], parent=list(parent),
+                      want_rows=True)
+    torch.cuda.synchronize()
+    assert "pooled thresholds" in ersd.ersd_last_launch()
+    check_verify(inp, out)
+
+
 def test_race_sample_draft_then_verify_is_consistent(ersd):
     """Drafting with race_sample and verifying with ersd_verify see the same draft winners."""
     w = wl.scaled(wl.CONFIGS["c2"], B=4)
