@@ -104,7 +104,8 @@ constexpr int kThreads = 128, kMinBlocks = 7;
 constexpr bool kMany = false;
 #include "ersd_kernel.inc"
 }  // namespace b128
-// The same two for calls with races that want several arrivals (tree and batch drafting, top_c > 1).
+// The same two for calls of few rows with races that want several arrivals (tree and batch
+// drafting, top_c > 1) and for every call with a race of more than 32 arrivals: see launch().
 namespace b256m {
 constexpr int kThreads = 256, kMinBlocks = 4;
 constexpr bool kMany = true;
