@@ -86,6 +86,7 @@ struct Params {
   uint32_t* near_tie;    // count of races with two consecutive arrivals closer than 1e-5 (nullable)
   int extra;             // 1 when near-ties are counted: every race is run for one more arrival
   int top_cmax;          // cluster kernel for several arrivals: most arrivals any race of the call wants
+  int top_split;         // the same kernel: 0, or 1 + the number of nodes with children when every row gets its own cluster
   Slot* slots;
 };
 
@@ -408,6 +409,8 @@ static int launch(const Params& p, const TreeDesc& tree, int dt, int cmax, cudaS
 constexpr int64_t kClusterAutoBlocksSample = 1280, kClusterAutoBlocksVerify = 768;
 // The same for races of several arrivals (ersd_cluster_top.inc; three blocks per SM).
 constexpr int64_t kClusterAutoBlocksTop = 600;
+// ... and the number of blocks up to which a tree's rows get a cluster each (one block per SM and a half)
+constexpr int64_t kClusterSplitBlocks = 384;
 constexpr size_t kClusterSmemBytes = 200 * 1024;  // dynamic shared memory a block of the cluster kernels may use
 
 // Tiles per block that fit (roles = rows raced together: 1, or 2 for a draft/target pair; cmax > 1:
@@ -527,15 +530,35 @@ template <int DT>
 static int launch_cluster_dt(const ersd_opts& o, const Params& p_in, const TreeDesc& tree, int cmax, cudaStream_t st) {
   Params p = p_in;
   p.top_cmax = cmax;
-  const int roles = (p.mode == kVerify && p.draft) ? 2 : 1;
+  int roles = (p.mode == kVerify && p.draft) ? 2 : 1;
   int CL = 1;
   const int ls = cluster_size(o, p, DT, cmax, &CL);
   if (ls != ERSD_OK) return ls;
   const int ntiles = (p.V + b256::kTile - 1) / b256::kTile;
+  // Trees of few positions: a cluster per ROW (a node's draft row and its target row side by side
+  // in two clusters, each drawing the position's race variables) while all clusters are resident
+  // at once; the longest chain of work in the call, the root's, is then half as long.
+  int jobs = p.rows;
+  if (cmax > 1 && roles == 2) {
+    int with_children = 0;
+    for (int n = 0; n < p.rows; ++n) with_children += tree.nchild[n] > 0 ? 1 : 0;
+    const int64_t rows_in_all = (int64_t)p.B * (p.rows + with_children);
+    bool split = rows_in_all * CL <= kClusterSplitBlocks;
+    if (!split && !o.split_v && CL >= 2 && rows_in_all * (CL / 2) <= kClusterSplitBlocks &&
+        (ntiles + CL / 2 - 1) / (CL / 2) <= cluster_max_tiles(DT, 1, cmax)) {
+      CL /= 2;  // (a row to a cluster of half as many blocks)
+      split = true;
+    }
+    if (split) {
+      p.top_split = 1 + with_children;
+      jobs = p.rows + with_children;
+      roles = 1;
+    }
+  }
   const int G = (ntiles + CL - 1) / CL;  // tiles per block; they fit, see cluster_applies
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
-  cfg.gridDim = dim3((unsigned)CL, (unsigned)p.rows, (unsigned)p.B);
+  cfg.gridDim = dim3((unsigned)CL, (unsigned)jobs, (unsigned)p.B);
   cfg.blockDim = dim3(b256::kThreads, 1, 1);
   cfg.dynamicSmemBytes = b256::cluster_role_bytes<DT>(G) * (size_t)roles + (cmax > 1 ? b256::top_list_bytes(cmax, CL) : 0);
   cfg.stream = st;
@@ -546,9 +569,9 @@ static int launch_cluster_dt(const ersd_opts& o, const Params& p_in, const TreeD
   at.val.clusterDim.z = 1;
   cfg.attrs = &at;
   cfg.numAttrs = 1;
-  snprintf(g_last_launch, sizeof g_last_launch, "%s<%s, %d row(s) per position>: clusters of %d x %d threads, %d positions",
-           cmax > 1 ? "ersd_cluster_top_kernel" : "ersd_cluster_kernel", DT == ERSD_BF16 ? "bf16" : "f32", roles, CL,
-           b256::kThreads, p.B * p.rows);
+  snprintf(g_last_launch, sizeof g_last_launch, "%s<%s, %d row(s) per cluster>: %d clusters of %d x %d threads, %d positions",
+           cmax > 1 ? "ersd_cluster_top_kernel" : "ersd_cluster_kernel", DT == ERSD_BF16 ? "bf16" : "f32", roles,
+           p.B * jobs, CL, b256::kThreads, p.B * p.rows);
   cudaError_t e;
   if (cmax > 1) {
     auto kernel = roles == 2 ? b256::ersd_cluster_top_kernel<DT, 2> : b256::ersd_cluster_top_kernel<DT, 1>;
