@@ -232,7 +232,7 @@ def test_small_trees_take_this_kernel_by_default(ersd):
     assert "ersd_cluster_top_kernel" in ersd.ersd_last_launch()
     assert "1 row(s) per cluster>: 10 clusters" in ersd.ersd_last_launch()   # root's draft row, nine target rows
     check_verify(inp, out)
-    mid = wl.scaled(wl.CONFIGS["c4"], B=4)                # 68 positions: draft and target row of a node in one cluster
+    mid = wl.scaled(wl.CONFIGS["c4"], B=4, V=128256)      # 68 positions: draft and target row of a node in one cluster
     inp = wl.make_inputs(mid)
     out = ersd.verify(inp["target"].cuda(), inp["draft"].cuda(), inp["seeds"].cuda(), inp["T"],
                       parent=list(inp["parent"]), want_rows=True)
