@@ -253,10 +253,7 @@ static int choose_threads(const ersd_opts& o, int64_t units, int* threads) {
   return ERSD_OK;
 }
 
-// Thread blocks per row.  At least one work item per resident-block slot, and two chunks per
-// row when rows are long: the hardware's block scheduler then evens out rows of different cost
-// and the last wave is made of half rows.  More chunks do not pay: each costs a block about as
-// much set-up, barrier and merge time as eight tiles of streaming (measured).
+// Thread blocks per row.
 static int choose_split(const ersd_opts& o, int64_t units, int V, int cmax, int threads) {
   int smax = kPartCap / cmax;
   if (smax > ERSD_MAX_SPLIT) smax = ERSD_MAX_SPLIT;
@@ -268,9 +265,16 @@ static int choose_split(const ersd_opts& o, int64_t units, int V, int cmax, int 
     S = (int)o.split_v;
     if (S > ntiles) S = ntiles;
   } else {
+    // about 1.7 blocks per SM: a block costs as much set-up, first threshold, merge and finish as
+    // eight tiles of streaming, so more chunks than the SMs need to be busy only add work
+    // (measured on calls of 48 to 400 rows: 5 to 15 % quicker than one block per resident slot)
     const int64_t slots = (int64_t)sm_count() * (threads == 128 ? b128::kMinBlocks : b256::kMinBlocks);
-    S = (int)((slots + units - 1) / units);
-    if (S < 2 && (int64_t)ntiles * tile >= 4 * kMinChunkTiles * b256::kTile) S = 2;
+    // (races of several arrivals: their rare path is the long one, and shorter chunks bound it;
+    // there a block per resident slot stays the better choice)
+    const int64_t wanted = cmax > 1 ? slots : ((int64_t)sm_count() * 27) / 16;
+    S = (int)((wanted + units - 1) / units);
+    // whole rows that make more than one wave, and rows of uneven cost (trees): halves even out the last wave
+    if (S < 2 && (units > slots || cmax > 1) && (int64_t)ntiles * tile >= 4 * kMinChunkTiles * b256::kTile) S = 2;
     const int by_v = ntiles / kMinChunkTiles;
     if (S > by_v) S = by_v;
   }
@@ -404,9 +408,10 @@ static int launch(const Params& p, const TreeDesc& tree, int dt, int cmax, cudaS
 // Latency path of calls of few rows: one cluster of thread blocks per position (ersd_cluster.inc).
 // ---------------------------------------------------------------------------------------------
 // Default choice: the cluster kernel is taken while its blocks number up to 1280 (sampling: 160
-// rows of 128256 logits) or 768 (verification: two rows per position; 96 positions); beyond that
-// the streaming kernel's throughput wins (measured at V = 128256 and 32000).
-constexpr int64_t kClusterAutoBlocksSample = 1280, kClusterAutoBlocksVerify = 768;
+// rows of 128256 logits) or, in verification (two rows per position), while the positions would
+// make up to 704 blocks in clusters of full size (44 positions of 128256 logits); beyond that the
+// streaming kernel's throughput wins (measured at V = 128256 and 32000).
+constexpr int64_t kClusterAutoBlocksSample = 1280, kClusterAutoBlocksVerify = 704;
 // The same for races of several arrivals (ersd_cluster_top.inc; three blocks per SM).
 constexpr int64_t kClusterAutoBlocksTop = 600;
 // ... and the number of blocks up to which a tree's rows get a cluster each (one block per SM and a half)
@@ -523,7 +528,15 @@ static bool cluster_by_default(const ersd_opts& o, const Params& p, int dt, int 
   if (cluster_size(o, p, dt, cmax, &CL) != ERSD_OK) return false;
   const int64_t blocks = (int64_t)p.B * p.rows * CL;
   if (cmax > 1) return blocks <= kClusterAutoBlocksTop;
-  return blocks <= (p.mode == kVerify ? kClusterAutoBlocksVerify : kClusterAutoBlocksSample);
+  if (p.mode == kVerify) {
+    // counted in clusters of the size a lone position would get (16 blocks at V = 128256, 4 at
+    // 32000), whatever size this call's clusters have: 44 and 176 positions at those two sizes
+    const int ntiles = (p.V + b256::kTile - 1) / b256::kTile;
+    int full = 1;
+    while (full < b256::kClusterMax && full * b256::kClusterGroups < ntiles) full *= 2;
+    return (int64_t)p.B * p.rows * full <= kClusterAutoBlocksVerify;
+  }
+  return blocks <= kClusterAutoBlocksSample;
 }
 
 template <int DT>
