@@ -90,6 +90,20 @@ def test_every_cluster_size_gives_the_same_arrivals(ersd):
         assert (tok == ref_tok).all() and (key == ref_key).all()
 
 
+def test_two_blocks_to_a_row_of_full_length(ersd):
+    """Two blocks to a row of 128256 logits and 32 arrivals wanted: 32 tiles to a block, hundreds of
+    groups on its list and a hundred survivors."""
+    B, V, c = 2, 128256, 32
+    g = torch.Generator().manual_seed(79)
+    logits = wl.zipf_rows(B, V, g, "cpu").view(B, 1, V).to(torch.bfloat16)
+    seeds = wl.make_seeds(73, 1, B)
+    tok, key = sample(ersd, logits, seeds, 1.0, c, CLUSTER, split_v=2)
+    assert "ersd_cluster_top_kernel" in ersd.ersd_last_launch()
+    assert check_sample(logits, seeds, 1.0, tok, key, c=c) == 0
+    tok_s, key_s = sample(ersd, logits, seeds, 1.0, c, STREAMING)
+    assert (tok == tok_s).all() and (key == key_s).all()
+
+
 def test_rows_with_fewer_tokens_than_arrivals_wanted(ersd):
     """Rows where fewer than c tokens have positive probability: the arrivals there are, then -1
     and +inf keys; a row of NaN or without any token gives no arrival at all."""
