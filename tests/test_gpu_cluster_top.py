@@ -139,6 +139,9 @@ def test_greedy_rows_of_tied_logits(ersd, V):
     assert t[1, 1].tolist() == list(range(V - 5, V)) + [0, 1, 2]
     tok_s, key_s = sample(ersd, logits, seeds, 0.0, c, STREAMING)
     assert (tok == tok_s).all() and (key == key_s).all()
+    if V > 100000:   # clusters of four: a block has more tied groups (4096) than its list holds and goes through all its indices
+        tok_4, key_4 = sample(ersd, logits, seeds, 0.0, c, CLUSTER, split_v=4)
+        assert (tok == tok_4).all() and (key == key_4).all()
 
 
 @pytest.mark.parametrize("c", [2, 4, 8, 32])
